@@ -1,0 +1,170 @@
+/*
+ * adadim.h - C ABI of the AdaDim layer-quantization library for NVIDIA B200 (sm_100a).
+ *
+ * The library quantizes one linear layer's weight W[out,in] to b-bit group-wise asymmetric
+ * integers under both grouping dimensions of the paper "Rethinking Channel Dimensions to
+ * Isolate Outliers for Low-bit Weight Quantization of LLMs" (arxiv 2309.15531): groups of g
+ * consecutive weights inside an output channel (a row of W, "per-OC", Section 2.1) and
+ * inside an input channel (a column of W, "per-IC", Section 3.2), scores both by the
+ * layer-output reconstruction error of Section 3.3, Eq. 1, and selects one.
+ *
+ * Conventions that hold for every entry point
+ *   - All matrices are row-major.  W[o,i] is at W + o*ldw + i; X[t,i] (token t) at X + t*ldx + i.
+ *   - Unless an argument is marked "host", every pointer is a DEVICE pointer owned by the
+ *     caller.  The library allocates no device memory and keeps no state between calls;
+ *     inputs are never modified.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream).  No entry point synchronizes; results are valid once the stream has run.
+ *   - The return value is an adadim_status.  Argument errors are found on the host before
+ *     anything is launched.  Conditions only the device can see (a non-positive Cholesky
+ *     pivot, a wait that ran out) are written to the caller's `status_dev` word, which the
+ *     call first sets to ADADIM_OK; kernels never trap.
+ *   - Non-finite weights or activations give unspecified codes (no error is raised).
+ */
+#ifndef ADADIM_H_
+#define ADADIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ADADIM_API __attribute__((visibility("default")))
+#else
+#define ADADIM_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ADADIM_OK = 0,
+  ADADIM_ERR_NULL = 1,       /* a required pointer is NULL                                  */
+  ADADIM_ERR_SHAPE = 2,      /* a size is negative or violates a divisibility rule          */
+  ADADIM_ERR_DTYPE = 3,      /* unknown element type for this argument                      */
+  ADADIM_ERR_PARAM = 4,      /* bits / group / dim / percdamp / blocksize out of range      */
+  ADADIM_ERR_ALIGN = 5,      /* pointer or leading dimension not 16-byte aligned            */
+  ADADIM_ERR_WORKSPACE = 6,  /* workspace smaller than adadim_workspace_bytes() says        */
+  ADADIM_ERR_NOT_PD = 7,     /* (device) damped Hessian is not positive definite            */
+  ADADIM_ERR_NUMERIC = 8,    /* (device) a reconstruction error is NaN                      */
+  ADADIM_ERR_TIMEOUT = 9,    /* (device) an internal wait exceeded its limit                */
+  ADADIM_ERR_CUDA = 10       /* a CUDA runtime / driver call failed                         */
+} adadim_status;
+
+typedef enum { ADADIM_F32 = 0, ADADIM_F16 = 1, ADADIM_BF16 = 2 } adadim_dtype;
+typedef enum { ADADIM_DIM_OC = 0, ADADIM_DIM_IC = 1, ADADIM_DIM_BOTH = 2 } adadim_dim;
+typedef enum { ADADIM_WS_HESSIAN = 0, ADADIM_WS_GPTQ = 1, ADADIM_WS_SCORE = 2,
+               ADADIM_WS_FACTOR = 3 } adadim_ws_kind;
+
+/*
+ * One quantized tensor (device pointers, caller-owned).
+ *   codes  [out][in*bits/32] uint32.  Code k of row o occupies bits [k*bits, (k+1)*bits) of
+ *          that row's little-endian stream of 32-bit words; the layout is the same for both
+ *          grouping dimensions.  (The paper fixes no packed format; its storage accounting,
+ *          Appendix C, counts bits only.)
+ *   scales fp16 bit patterns.  per-OC: [out][in/g];  per-IC: [out/g][in]   (Section 3.2).
+ *   zeros  fp16 bit patterns holding the integer zero point 0..2^bits-1, same shape.
+ * Dequantized weight: q = scale * (code - zero).
+ */
+typedef struct {
+  uint32_t* codes;
+  uint16_t* scales;
+  uint16_t* zeros;
+} adadim_qtensor;
+
+/*
+ * Calibration Hessian  H += 2 * X^T X  over one chunk of tokens (Section 4.4: the inverse
+ * Hessian GPTQ uses is "formed by activations"; Section 2.2).
+ *   X        [n_tokens][in], xdtype ADADIM_BF16 (tcgen05 tensor-core path) or ADADIM_F32.
+ *            ldx in elements; X and ldx*sizeof(elem) must be 16-byte aligned.
+ *   H        [in][in] fp32, in/out: the caller zeroes it before the first chunk.  Both
+ *            triangles are updated.  in must be a multiple of 8.
+ *   n_seen   host pointer, in/out, may be NULL: incremented by n_tokens.
+ *   status_dev  device int, may be NULL.
+ *   workspace   unused by the current kernels (adadim_workspace_bytes(ADADIM_WS_HESSIAN,..)
+ *               is 0); may be NULL.
+ */
+ADADIM_API int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_tokens, int64_t in, int64_t ldx,
+                              float* H, int64_t* n_seen, int* status_dev,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Round-to-nearest group quantizer (Section 4.1: uniform asymmetric, group size g; Appendix A.2:
+ * min-max), in one pass over W for one or both grouping dimensions (Section 3.3: the weights are
+ * quantized independently per-IC and per-OC).  Per group G, in IEEE binary32:
+ *     lo = min(0, min_G w)   hi = max(0, max_G w)
+ *     s  = fp16_rn((hi - lo) / maxq);   if s == 0 or s is not finite: s = 1, z = 0, codes 0
+ *     z  = clamp(rint(-lo / s), 0, maxq)
+ *     c  = clamp(rint(w / s) + z, 0, maxq)          maxq = 2^bits - 1, rint = ties to even
+ *   W      [out][in], wdtype ADADIM_F16 or ADADIM_F32; ldw in elements, 16-byte aligned rows.
+ *   bits   3 or 4;  group 32, 64 or 128.
+ *   dim    ADADIM_DIM_OC (q_oc written), ADADIM_DIM_IC (q_ic written) or ADADIM_DIM_BOTH.
+ *   Shape rules: in % 32 == 0; per-OC needs in % group == 0; per-IC needs out % group == 0.
+ *   out == 0 or in == 0 is accepted and does nothing.
+ */
+ADADIM_API int adadim_quantize_rtn(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
+                        int bits, int group, int dim,
+                        const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, void* cuda_stream);
+
+/*
+ * Damped Cholesky-inverse factor used by GPTQ (Section 2.2; the damping is the published
+ * algorithm's): columns with H[i,i] == 0 get H[i,i] = 1 ("dead" columns), then
+ *     Hd = H + lambda*I,  lambda = percdamp * mean(diag H),   U upper triangular, Hd^-1 = U^T U.
+ *   H  [in][in] fp32 (not modified);  U [in][in] fp32 out, strictly-lower part set to 0.
+ *   in must be a multiple of 64.
+ *   workspace  adadim_workspace_bytes(ADADIM_WS_FACTOR, 0, in, 0, 0) bytes, 256-byte aligned.
+ *   status_dev ADADIM_ERR_NOT_PD if a pivot is not positive.
+ */
+ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, float percdamp, float* U,
+                                   int* status_dev, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream);
+
+/*
+ * GPTQ (Section 2.2; Section 3.3: the per-IC variant changes only the quantization step):
+ * columns are quantized in order; after column i the rounding error e = (w_i - q_i) / U[i,i]
+ * is propagated to the not-yet-quantized columns, W[:, j] -= e * U[i, j] (j > i), lazily
+ * batched in blocks of `blocksize` columns.  Group parameters come from the CURRENT
+ * (already compensated) weights with the formula of adadim_quantize_rtn: per-OC at each
+ * group's first column, from that group's columns; per-IC at every column, from its g-row
+ * groups.  Weights of dead columns are treated as 0.
+ *   H          [in][in] fp32, used when U == NULL (the factor is then computed into workspace).
+ *   U          optional precomputed adadim_cholesky_inverse_factor of the same H, or NULL.
+ *   blocksize  128.  group must divide 128.  in % 128 == 0, out % 128 == 0.
+ *   gptq_loss  optional device double[2] (OC, IC): 1/2 * sum of e^2.
+ *   workspace  adadim_workspace_bytes(ADADIM_WS_GPTQ, out, in, bits, group), 256-byte aligned.
+ */
+ADADIM_API int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
+                         const float* H, const float* U, int bits, int group, int dim,
+                         float percdamp, int blocksize,
+                         const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+                         double* gptq_loss, int* status_dev,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Reconstruction error of both quantized tensors and the selection (Section 3.3, Eq. 1;
+ * Appendix B):  E_dim = || X (W - Q_dim)^T ||_F^2 = 1/2 trace((W - Q_dim) H (W - Q_dim)^T)
+ * with the undamped H = 2 X^T X;  chosen = IC iff E_ic < E_oc (ties and NaN give OC, the
+ * dimension evaluated first).
+ *   err     device double[2] = {E_oc, E_ic};  chosen  device int (adadim_dim).
+ *   Either q_oc or q_ic may be NULL: its error is reported as +infinity.
+ *   in % 64 == 0, out % 128 == 0.
+ *   workspace  adadim_workspace_bytes(ADADIM_WS_SCORE, out, in, bits, group), 256-byte aligned.
+ */
+ADADIM_API int adadim_score_select(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
+                        const float* H, int bits, int group,
+                        const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+                        double* err, int* chosen, int* status_dev,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Helpers. */
+ADADIM_API size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int group);
+/* Unpack the bitstream format above: dst [out][in] uint8 (device). */
+ADADIM_API int adadim_unpack_codes(const uint32_t* codes, int64_t out, int64_t in, int bits, uint8_t* dst,
+                        void* cuda_stream);
+ADADIM_API const char* adadim_strerror(int status);
+ADADIM_API int adadim_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADADIM_H_ */

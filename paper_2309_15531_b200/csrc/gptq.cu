@@ -1,0 +1,343 @@
+// GPTQ with lazily batched error compensation (paper Section 2.2; Section 3.3: the per-IC
+// variant changes only the quantization step).  Columns are handled in blocks of 128:
+//   block kernel    - one CTA per 128-row slab and grouping dimension walks the block's
+//                     columns in order: group parameters from the current weights, code,
+//                     error e = (w - q) / U[i,i], and the update of the block's remaining
+//                     columns, w[j] -= e U[i,j].  The slab lives in shared memory; the 32
+//                     columns being worked on live in registers.
+//   trailing kernel - W[:, after the block] -= Err[out,128] * U[block rows, after the block],
+//                     an fp32 FFMA matrix product (the update feeds rounding decisions, so it
+//                     keeps full fp32 products).
+// Rows are independent under per-OC grouping; under per-IC grouping a group couples g
+// consecutive rows of one column, which is why a CTA owns a whole 128-row slab.
+#include "common.cuh"
+
+namespace adadim {
+
+size_t factor_workspace_bytes(int64_t n);
+int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
+                  cudaStream_t st);
+
+namespace {
+
+constexpr int kBlk = 128;            // lazy-batch block width (columns) and slab height (rows)
+constexpr int kSub = 32;             // columns held in registers at a time
+constexpr int kPad = kBlk + 1;       // shared-memory row pitch (floats): conflict-free column access
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const float* __restrict__ H, int ndim,
+            float* __restrict__ Wc) {
+  int64_t e = (static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x) * 8;
+  if (e >= out * in) return;
+  int64_t o = e / in, i = e % in;
+  float v[8];
+  load8(W + o * ldw + i, v);
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+    if (H[(i + k) * in + (i + k)] == 0.0f) v[k] = 0.0f;        // dead column
+  for (int d = 0; d < ndim; ++d) {
+    float4* dst = reinterpret_cast<float4*>(Wc + static_cast<int64_t>(d) * out * in + e);
+    dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+    dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+struct BlockArgs {
+  float* Wc;                 // [ndim][out][in] working weights
+  const float* U;            // [in][in]
+  float* Err;                // [ndim][out][128]
+  double* loss_part;         // [ndim][out/128]
+  adadim_qtensor q[2];       // outputs for the dimension(s) in flight
+  int dim_of[2];             // grouping dimension of working copy d
+  int64_t out, in;
+  int i1;                    // first column of the block
+};
+
+template <int BITS, int G>
+__global__ void __launch_bounds__(kBlk, 1)
+block_kernel(const BlockArgs a) {
+  constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr int NG = kBlk / G;                       // per-IC groups in the slab
+  extern __shared__ float sm[];
+  float* Ws = sm;                                    // [128][129] slab of the working weights
+  float* Us = Ws + kBlk * kPad;                      // [128][128] block of U (upper triangle used)
+  float* Es = Us + kBlk * kBlk;                      // [128][129] errors
+  float* invd = Es + kBlk * kPad;                    // [128] 1 / U[i,i]
+  float* red = invd + kBlk;                          // [2][4][2] per-IC min / max exchange
+  uint16_t* Ss = reinterpret_cast<uint16_t*>(red + 16);   // [NG][128] per-IC scales (fp16 bits)
+  uint16_t* Zs = Ss + NG * kBlk;                          // [NG][128]
+
+  const int d = blockIdx.y;
+  const bool is_ic = a.dim_of[d] == ADADIM_DIM_IC;
+  const adadim_qtensor q = a.q[d];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kBlk;
+  const int64_t row = row0 + tid;
+  float* Wd = a.Wc + static_cast<int64_t>(d) * a.out * a.in;
+
+  // stage the slab and the U block (coalesced), then work row-per-thread
+  for (int e = tid; e < kBlk * kBlk / 4; e += kBlk) {
+    int r = e >> 5, c4 = (e & 31) * 4;
+    float4 w = *reinterpret_cast<const float4*>(Wd + (row0 + r) * a.in + a.i1 + c4);
+    Ws[r * kPad + c4 + 0] = w.x; Ws[r * kPad + c4 + 1] = w.y; Ws[r * kPad + c4 + 2] = w.z; Ws[r * kPad + c4 + 3] = w.w;
+    *reinterpret_cast<float4*>(Us + r * kBlk + c4) =
+        *reinterpret_cast<const float4*>(a.U + static_cast<int64_t>(a.i1 + r) * a.in + a.i1 + c4);
+  }
+  __syncthreads();
+  invd[tid] = 1.0f / Us[tid * kBlk + tid];
+  __syncthreads();
+
+  float* wrow = Ws + tid * kPad;
+  float* erow = Es + tid * kPad;
+  GroupParams gp = {1.0f, 0.0f, 0.0f};
+  double loss = 0.0;
+
+#pragma unroll 1
+  for (int sb = 0; sb < kBlk / kSub; ++sb) {
+    const int cbase = sb * kSub;
+    float w[kSub], err[kSub];
+    uint32_t cw[BITS] = {};
+#pragma unroll
+    for (int k = 0; k < kSub; ++k) w[k] = wrow[cbase + k];
+
+#pragma unroll
+    for (int ii = 0; ii < kSub; ++ii) {
+      const int i = cbase + ii;                      // column inside the block
+      if (!is_ic) {
+        if ((ii % G) == 0 && (cbase % G) == 0) {     // per-OC: parameters at the group's first column
+          float mn = w[ii], mx = w[ii];
+          if (G == kSub) {
+#pragma unroll
+            for (int k = 1; k < kSub; ++k) { mn = fminf(mn, w[k]); mx = fmaxf(mx, w[k]); }
+          } else {
+            for (int k = 1; k < G; ++k) { float v = wrow[i + k]; mn = fminf(mn, v); mx = fmaxf(mx, v); }
+          }
+          gp = group_params(mn, mx, maxq);
+          int64_t idx = row * (a.in / G) + (a.i1 + i) / G;
+          q.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
+          q.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
+        }
+      } else {                                       // per-IC: parameters of this column's g-row groups
+        float mn = w[ii], mx = w[ii];
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+          mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, m));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+        }
+        if (G > 32) {
+          float* slot = red + (ii & 1) * 8;
+          if (lane == 0) { slot[warp * 2] = mn; slot[warp * 2 + 1] = mx; }
+          __syncthreads();
+          constexpr int WPG = G / 32;                // warps per group
+          const int w0 = (warp / WPG) * WPG;
+          mn = slot[w0 * 2]; mx = slot[w0 * 2 + 1];
+#pragma unroll
+          for (int k = 1; k < WPG; ++k) { mn = fminf(mn, slot[(w0 + k) * 2]); mx = fmaxf(mx, slot[(w0 + k) * 2 + 1]); }
+        }
+        gp = group_params(mn, mx, maxq);
+        if ((tid % G) == 0) {
+          Ss[(tid / G) * kBlk + i] = __half_as_ushort(__float2half_rn(gp.s));
+          Zs[(tid / G) * kBlk + i] = __half_as_ushort(__float2half_rn(gp.z));
+        }
+      }
+      const int c = code_of(quotient(w[ii], gp.s, gp.rcp), gp.z, maxq);
+      const float qv = __fmul_rn(gp.s, static_cast<float>(c) - gp.z);
+      const float e = (w[ii] - qv) * invd[i];
+      err[ii] = e;
+      erow[i] = e;
+      loss += static_cast<double>(e) * static_cast<double>(e);
+      {
+        const int bit = ii * BITS, wi = bit >> 5, sh = bit & 31;
+        cw[wi] |= static_cast<uint32_t>(c) << sh;
+        if (sh + BITS > 32) cw[wi + 1] |= static_cast<uint32_t>(c) >> (32 - sh);
+      }
+      const float* urow = Us + i * kBlk + cbase;
+#pragma unroll
+      for (int jj = ii + 1; jj < kSub; ++jj) w[jj] = fmaf(-e, urow[jj], w[jj]);
+    }
+    // codes of these 32 columns: BITS whole words of this row's bitstream
+    uint32_t* cdst = q.codes + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) cdst[k] = cw[k];
+    // lazy update of the block's later columns with this sub-block's 32 errors
+#pragma unroll 1
+    for (int jc = cbase + kSub; jc < kBlk; jc += kSub) {
+      float acc[kSub];
+#pragma unroll
+      for (int k = 0; k < kSub; ++k) acc[k] = wrow[jc + k];
+#pragma unroll
+      for (int ii = 0; ii < kSub; ++ii) {
+        const float4* u4 = reinterpret_cast<const float4*>(Us + (cbase + ii) * kBlk + jc);
+#pragma unroll
+        for (int k4 = 0; k4 < kSub / 4; ++k4) {
+          float4 u = u4[k4];
+          acc[k4 * 4 + 0] = fmaf(-err[ii], u.x, acc[k4 * 4 + 0]);
+          acc[k4 * 4 + 1] = fmaf(-err[ii], u.y, acc[k4 * 4 + 1]);
+          acc[k4 * 4 + 2] = fmaf(-err[ii], u.z, acc[k4 * 4 + 2]);
+          acc[k4 * 4 + 3] = fmaf(-err[ii], u.w, acc[k4 * 4 + 3]);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kSub; ++k) wrow[jc + k] = acc[k];
+    }
+  }
+
+  // ---- outputs: errors (coalesced), per-IC parameters, loss ------------------------------
+  __syncthreads();
+  float* Ed = a.Err + (static_cast<int64_t>(d) * a.out + row0) * kBlk;
+  for (int e = tid; e < kBlk * kBlk; e += kBlk) Ed[e] = Es[(e >> 7) * kPad + (e & 127)];
+  if (is_ic) {
+    for (int e = tid; e < NG * kBlk; e += kBlk) {
+      int64_t idx = (row0 / G + e / kBlk) * a.in + a.i1 + (e % kBlk);
+      q.scales[idx] = Ss[e];
+      q.zeros[idx] = Zs[e];
+    }
+  }
+  __shared__ double lred[kBlk / 32];
+  for (int m = 16; m > 0; m >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, m);
+  if (lane == 0) lred[warp] = loss;
+  __syncthreads();
+  if (tid == 0) a.loss_part[static_cast<int64_t>(d) * (a.out / kBlk) + blockIdx.x] += (lred[0] + lred[1]) + (lred[2] + lred[3]);
+}
+
+// Wc[d][:, c0 + ...] -= Err[d] * U[i1 .. i1+127, c0 + ...], 128 x 128 output tile per CTA.
+__global__ void __launch_bounds__(256)
+trailing_kernel(float* __restrict__ Wc, const float* __restrict__ U, const float* __restrict__ Err, int64_t out,
+                int64_t in, int i1) {
+  __shared__ float sa[8][kBlk + 4];     // Err^T slice: [k][row]
+  __shared__ float sb[8][kBlk + 4];     // U slice:     [k][col]
+  const int64_t c0 = static_cast<int64_t>(i1) + kBlk + static_cast<int64_t>(blockIdx.x) * kBlk;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kBlk;
+  float* Wd = Wc + static_cast<int64_t>(blockIdx.z) * out * in;
+  const float* Ed = Err + (static_cast<int64_t>(blockIdx.z) * out + r0) * kBlk;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  float acc[8][8] = {};
+  for (int k0 = 0; k0 < kBlk; k0 += 8) {
+    {
+      // Err tile: 128 rows x 8 k -> transposed; 256 threads x 4 elements
+      const int r = threadIdx.x >> 1, kq = (threadIdx.x & 1) * 4;
+      float4 v = *reinterpret_cast<const float4*>(Ed + r * kBlk + k0 + kq);
+      sa[kq + 0][r] = v.x; sa[kq + 1][r] = v.y; sa[kq + 2][r] = v.z; sa[kq + 3][r] = v.w;
+      const int kk = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4;
+      *reinterpret_cast<float4*>(&sb[kk][c4]) =
+          *reinterpret_cast<const float4*>(U + static_cast<int64_t>(i1 + k0 + kk) * in + c0 + c4);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      float av[8], bv[8];
+      *reinterpret_cast<float4*>(av) = *reinterpret_cast<const float4*>(&sa[kk][ty * 4]);
+      *reinterpret_cast<float4*>(av + 4) = *reinterpret_cast<const float4*>(&sa[kk][64 + ty * 4]);
+      *reinterpret_cast<float4*>(bv) = *reinterpret_cast<const float4*>(&sb[kk][tx * 4]);
+      *reinterpret_cast<float4*>(bv + 4) = *reinterpret_cast<const float4*>(&sb[kk][64 + tx * 4]);
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+#pragma unroll
+        for (int n = 0; n < 8; ++n) acc[m][n] = fmaf(av[m], bv[n], acc[m][n]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int m = 0; m < 8; ++m) {
+    const int64_t r = r0 + (m < 4 ? ty * 4 + m : 64 + ty * 4 + (m - 4));
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float4* p = reinterpret_cast<float4*>(Wd + r * in + c0 + h * 64 + tx * 4);
+      float4 v = *p;
+      v.x -= acc[m][h * 4 + 0]; v.y -= acc[m][h * 4 + 1]; v.z -= acc[m][h * 4 + 2]; v.w -= acc[m][h * 4 + 3];
+      *p = v;
+    }
+  }
+}
+
+__global__ void loss_kernel(const double* __restrict__ part, int ndim, int slabs, BlockArgs a, double* loss_out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    loss_out[0] = 0.0; loss_out[1] = 0.0;
+    for (int d = 0; d < ndim; ++d) {
+      double s = 0.0;
+      for (int k = 0; k < slabs; ++k) s += part[d * slabs + k];
+      loss_out[a.dim_of[d]] = 0.5 * s;
+    }
+  }
+}
+
+constexpr size_t block_smem_bytes() {
+  return (kBlk * kPad * 2 + kBlk * kBlk + kBlk + 16) * sizeof(float) + 2 * 4 * kBlk * sizeof(uint16_t);
+}
+
+template <int BITS, int G>
+int block_launch(const BlockArgs& a, int slabs, int ndim, cudaStream_t st) {
+  ADADIM_CUDA_TRY(cudaFuncSetAttribute(block_kernel<BITS, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(block_smem_bytes())));
+  block_kernel<BITS, G><<<dim3(slabs, ndim), kBlk, block_smem_bytes(), st>>>(a);
+  return ADADIM_OK;
+}
+
+struct GptqLayout { size_t wc_off, err_off, loss_off, u_off, factor_off, total; };
+GptqLayout gptq_layout(int64_t out, int64_t in) {
+  GptqLayout L;
+  size_t off = 0;
+  L.wc_off = off;     off += round_up(static_cast<size_t>(2) * out * in * 4, 256);
+  L.err_off = off;    off += round_up(static_cast<size_t>(2) * out * kBlk * 4, 256);
+  L.loss_off = off;   off += round_up(static_cast<size_t>(2) * (out / kBlk + 1) * 8, 256);
+  L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 4, 256);
+  L.factor_off = off; off += factor_workspace_bytes(in);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+size_t gptq_workspace_bytes(int64_t out, int64_t in) { return gptq_layout(out, in).total; }
+
+int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const float* U_in,
+                int bits, int group, int dim, float percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st) {
+  GptqLayout L = gptq_layout(out, in);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  BlockArgs a = {};
+  a.Wc = reinterpret_cast<float*>(ws + L.wc_off);
+  a.Err = reinterpret_cast<float*>(ws + L.err_off);
+  a.loss_part = reinterpret_cast<double*>(ws + L.loss_off);
+  a.out = out;
+  a.in = in;
+  int ndim = 0;
+  if (dim == ADADIM_DIM_OC || dim == ADADIM_DIM_BOTH) { a.q[ndim] = *q_oc; a.dim_of[ndim] = ADADIM_DIM_OC; ++ndim; }
+  if (dim == ADADIM_DIM_IC || dim == ADADIM_DIM_BOTH) { a.q[ndim] = *q_ic; a.dim_of[ndim] = ADADIM_DIM_IC; ++ndim; }
+
+  const float* U = U_in;
+  if (U == nullptr) {
+    float* Uw = reinterpret_cast<float*>(ws + L.u_off);
+    int rc = factor_launch(H, in, percdamp, Uw, status_dev, ws + L.factor_off, st);
+    if (rc != ADADIM_OK) return rc;
+    U = Uw;
+  }
+  a.U = U;
+
+  const unsigned ib = static_cast<unsigned>((out * in / 8 + 255) / 256);
+  if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, ndim, a.Wc);
+  else init_kernel<<<ib, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, H, ndim, a.Wc);
+  ADADIM_CUDA_TRY(cudaMemsetAsync(a.loss_part, 0, static_cast<size_t>(2) * (out / kBlk + 1) * 8, st));
+
+  const int slabs = static_cast<int>(out / kBlk);
+  for (int i1 = 0; i1 < in; i1 += kBlk) {
+    a.i1 = i1;
+    int rc;
+    if (bits == 3) {
+      rc = group == 128 ? block_launch<3, 128>(a, slabs, ndim, st) : group == 64 ? block_launch<3, 64>(a, slabs, ndim, st)
+                                                                                 : block_launch<3, 32>(a, slabs, ndim, st);
+    } else {
+      rc = group == 128 ? block_launch<4, 128>(a, slabs, ndim, st) : group == 64 ? block_launch<4, 64>(a, slabs, ndim, st)
+                                                                                 : block_launch<4, 32>(a, slabs, ndim, st);
+    }
+    if (rc != ADADIM_OK) return rc;
+    const int64_t rest = in - i1 - kBlk;
+    if (rest > 0)
+      trailing_kernel<<<dim3(static_cast<unsigned>(rest / kBlk), slabs, ndim), 256, 0, st>>>(a.Wc, U, a.Err, out, in, i1);
+  }
+  if (gptq_loss != nullptr) loss_kernel<<<1, 32, 0, st>>>(a.loss_part, ndim, slabs, a, gptq_loss);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+}  // namespace adadim

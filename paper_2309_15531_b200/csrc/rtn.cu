@@ -1,0 +1,244 @@
+// Round-to-nearest group quantizer for both grouping dimensions in one pass over W
+// (paper Section 3.3: the weights are quantized per-OC and per-IC independently; Section 4.1:
+// uniform asymmetric, group size g).  A 128 x 128 tile of W holds whole per-OC groups (row
+// segments) and whole per-IC groups (column segments) for every supported g, so one CTA reads
+// its tile once, keeps it in registers and emits codes and parameters for both dimensions.
+// The kernel is bound by HBM traffic: per weight it reads sizeof(T) bytes and writes, per
+// dimension, bits/8 bytes of codes and 4/g bytes of parameters.
+#include "common.cuh"
+
+namespace adadim {
+namespace {
+
+constexpr int kThreads = 256;       // 16 threads across a tile row (8 columns each) x 16 rows
+constexpr int kPasses = 8;          // 16 rows per pass
+
+// Pack eight codes (column order) of `BITS` bits and hand back this thread's share of the
+// row's bitstream.  acc arrives as sum_k(tbits_k << BITS*k) - bias, i.e. the packed value.
+template <int BITS>
+__device__ __forceinline__ void store_codes(uint32_t packed, uint32_t* row_words, int colvec, bool ok) {
+  if (BITS == 4) {
+    if (ok) row_words[colvec] = packed;
+  } else {  // BITS == 3: 24 bits per thread, four threads make three words
+    uint32_t up = __shfl_down_sync(0xffffffffu, packed, 1);
+    int k = colvec & 3;
+    uint32_t word = (packed >> (8 * k)) | (up << (24 - 8 * k));
+    if (ok && k < 3) row_words[(colvec >> 2) * 3 + k] = word;
+  }
+}
+
+template <typename T, int BITS, int G, bool DO_OC, bool DO_IC>
+__global__ void __launch_bounds__(kThreads, 2)
+rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
+                adadim_qtensor qoc, adadim_qtensor qic) {
+  constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr int NG = kTile / G;               // per-IC groups stacked in one tile
+  constexpr int PPG = kPasses / NG;           // passes per such group
+  constexpr int LANES_PER_OCG = G / 8;        // threads sharing one per-OC group
+  constexpr uint32_t kOnes = BITS == 3 ? 0x00249249u : 0x11111111u;   // sum_k 1 << BITS*k
+
+  __shared__ float s_mn[NG][8][kTile];
+  __shared__ float s_mx[NG][8][kTile];
+  __shared__ float s_s[NG][kTile];
+  __shared__ float s_z[NG][kTile];
+
+  const int tid = threadIdx.x;
+  const int colvec = tid & 15, rowsub = tid >> 4;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kTile;
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * kTile;
+  const int64_t col = c0 + colvec * 8;
+  const bool col_ok = col < in;               // in % 32 == 0: a thread's 8 columns are all in or out
+  const int64_t words_per_row = in * BITS / 32;
+
+  float w[kPasses][8];
+#pragma unroll
+  for (int p = 0; p < kPasses; ++p) {
+    int64_t row = r0 + p * 16 + rowsub;
+    if (col_ok && row < out) {
+      load8(W + row * ldw + col, w[p]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) w[p][k] = 0.0f;     // neutral: 0 always lies inside [lo, hi]
+    }
+  }
+
+  // ---- per-IC statistics: column minima / maxima over each g-row group of the tile ---------
+  if (DO_IC) {
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      float mn[8], mx[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { mn[k] = w[gi * PPG][k]; mx[k] = mn[k]; }
+#pragma unroll
+      for (int p = 1; p < PPG; ++p)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          mn[k] = fminf(mn[k], w[gi * PPG + p][k]);
+          mx[k] = fmaxf(mx[k], w[gi * PPG + p][k]);
+        }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        mn[k] = fminf(mn[k], __shfl_xor_sync(0xffffffffu, mn[k], 16));
+        mx[k] = fmaxf(mx[k], __shfl_xor_sync(0xffffffffu, mx[k], 16));
+      }
+      if (lane < 16) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          s_mn[gi][warp][colvec * 8 + k] = mn[k];
+          s_mx[gi][warp][colvec * 8 + k] = mx[k];
+        }
+      }
+    }
+    __syncthreads();
+    for (int t = tid; t < NG * kTile; t += kThreads) {
+      int gi = t / kTile, c = t % kTile;
+      float mn = s_mn[gi][0][c], mx = s_mx[gi][0][c];
+#pragma unroll
+      for (int wv = 1; wv < 8; ++wv) {
+        mn = fminf(mn, s_mn[gi][wv][c]);
+        mx = fmaxf(mx, s_mx[gi][wv][c]);
+      }
+      GroupParams gp = group_params(mn, mx, maxq);
+      s_s[gi][c] = gp.rcp == 0.0f ? 0.0f : gp.s;      // 0 marks a degenerate group
+      s_z[gi][c] = gp.z;
+      int64_t grow = r0 / G + gi;
+      if (c0 + c < in && grow * G < out) {
+        qic.scales[grow * in + c0 + c] = __half_as_ushort(__float2half_rn(gp.s));
+        qic.zeros[grow * in + c0 + c] = __half_as_ushort(__float2half_rn(gp.z));
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- codes ------------------------------------------------------------------------------
+#pragma unroll
+  for (int gi = 0; gi < NG; ++gi) {
+    float ic_s[8], ic_r[8], ic_z[8];
+    uint32_t ic_bias = 0;
+    if (DO_IC) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        float s = s_s[gi][colvec * 8 + k];
+        ic_z[k] = s_z[gi][colvec * 8 + k];
+        ic_r[k] = s == 0.0f ? 0.0f : __frcp_rn(s);
+        ic_s[k] = s == 0.0f ? 1.0f : s;
+        ic_bias += static_cast<uint32_t>(kRoundMagicBits - static_cast<int>(ic_z[k])) << (BITS * k);
+      }
+    }
+#pragma unroll
+    for (int pp = 0; pp < PPG; ++pp) {
+      const int p = gi * PPG + pp;
+      const int64_t row = r0 + p * 16 + rowsub;
+      const bool ok = col_ok && row < out;
+      if (DO_OC) {
+        float mn = w[p][0], mx = w[p][0];
+#pragma unroll
+        for (int k = 1; k < 8; ++k) { mn = fminf(mn, w[p][k]); mx = fmaxf(mx, w[p][k]); }
+#pragma unroll
+        for (int m = 1; m < LANES_PER_OCG; m <<= 1) {
+          mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, m));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+        }
+        GroupParams gp = group_params(mn, mx, maxq);
+        if (ok && (colvec % LANES_PER_OCG) == 0) {
+          int64_t idx = row * (in / G) + col / G;
+          qoc.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
+          qoc.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
+        }
+        uint32_t acc = 0;
+        const float zlo = kRoundMagic - gp.z, zhi = kRoundMagic + (maxq - gp.z);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          float t = __fadd_rn(quotient(w[p][k], gp.s, gp.rcp), kRoundMagic);
+          t = fminf(fmaxf(t, zlo), zhi);
+          acc += static_cast<uint32_t>(__float_as_int(t)) << (BITS * k);
+        }
+        acc -= static_cast<uint32_t>(kRoundMagicBits - static_cast<int>(gp.z)) * kOnes;
+        store_codes<BITS>(acc, qoc.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
+      }
+      if (DO_IC) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          float t = __fadd_rn(quotient(w[p][k], ic_s[k], ic_r[k]), kRoundMagic);
+          t = fminf(fmaxf(t, kRoundMagic - ic_z[k]), kRoundMagic + (maxq - ic_z[k]));
+          acc += static_cast<uint32_t>(__float_as_int(t)) << (BITS * k);
+        }
+        acc -= ic_bias;
+        store_codes<BITS>(acc, qic.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
+      }
+    }
+  }
+}
+
+template <typename T, int BITS, int G>
+void launch_dims(const T* W, int64_t out, int64_t in, int64_t ldw, int dim,
+                 const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  dim3 grid(static_cast<unsigned>((in + kTile - 1) / kTile), static_cast<unsigned>((out + kTile - 1) / kTile));
+  if (dim == ADADIM_DIM_BOTH)
+    rtn_tile_kernel<T, BITS, G, true, true><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+  else if (dim == ADADIM_DIM_OC)
+    rtn_tile_kernel<T, BITS, G, true, false><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+  else
+    rtn_tile_kernel<T, BITS, G, false, true><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+}
+
+template <typename T, int BITS>
+void launch_group(const T* W, int64_t out, int64_t in, int64_t ldw, int group, int dim,
+                  const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  if (group == 128) launch_dims<T, BITS, 128>(W, out, in, ldw, dim, qoc, qic, st);
+  else if (group == 64) launch_dims<T, BITS, 64>(W, out, in, ldw, dim, qoc, qic, st);
+  else launch_dims<T, BITS, 32>(W, out, in, ldw, dim, qoc, qic, st);
+}
+
+template <int BITS>
+__global__ void unpack_kernel(const uint32_t* __restrict__ codes, int64_t out, int64_t in, uint8_t* __restrict__ dst) {
+  // one thread per 32 codes (BITS words of input, 32 bytes of output)
+  int64_t chunks_per_row = in / 32;
+  int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t >= out * chunks_per_row) return;
+  int64_t row = t / chunks_per_row, ch = t % chunks_per_row;
+  const uint32_t* src = codes + row * (in * BITS / 32) + ch * BITS;
+  uint32_t wds[BITS + 1];
+#pragma unroll
+  for (int k = 0; k < BITS; ++k) wds[k] = src[k];
+  wds[BITS] = 0;
+  uint32_t outw[8];
+#pragma unroll
+  for (int k = 0; k < 32; ++k) {
+    int bit = k * BITS, wi = bit >> 5, sh = bit & 31;
+    uint32_t v = wds[wi] >> sh;
+    if (sh + BITS > 32) v |= wds[wi + 1] << (32 - sh);
+    v &= (1u << BITS) - 1u;
+    if ((k & 3) == 0) outw[k >> 2] = v; else outw[k >> 2] |= v << (8 * (k & 3));
+  }
+  uint4* d = reinterpret_cast<uint4*>(dst + row * in + ch * 32);
+  d[0] = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+  d[1] = make_uint4(outw[4], outw[5], outw[6], outw[7]);
+}
+
+}  // namespace
+
+int rtn_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, int bits, int group, int dim,
+               const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  if (wdtype == ADADIM_F16) {
+    if (bits == 3) launch_group<__half, 3>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
+    else launch_group<__half, 4>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
+  } else {
+    if (bits == 3) launch_group<float, 3>(static_cast<const float*>(W), out, in, ldw, group, dim, qoc, qic, st);
+    else launch_group<float, 4>(static_cast<const float*>(W), out, in, ldw, group, dim, qoc, qic, st);
+  }
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+int unpack_launch(const uint32_t* codes, int64_t out, int64_t in, int bits, uint8_t* dst, cudaStream_t st) {
+  int64_t n = out * (in / 32);
+  if (n == 0) return ADADIM_OK;
+  unsigned blocks = static_cast<unsigned>((n + 255) / 256);
+  if (bits == 3) unpack_kernel<3><<<blocks, 256, 0, st>>>(codes, out, in, dst);
+  else unpack_kernel<4><<<blocks, 256, 0, st>>>(codes, out, in, dst);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+}  // namespace adadim

@@ -1,0 +1,421 @@
+// Tensor-core kernels (tcgen05 MMA, TMEM accumulators, TMA-fed shared-memory ring):
+//   * calibration Hessian  H += 2 X^T X  (paper Section 4.4; Section 2.2) as a symmetric
+//     rank-k update over the tokens, lower-triangle 256 x 256 output tiles only;
+//   * the reconstruction-error contraction  S = D H  of  1/2 trace(D H D^T)  (Section 3.3, Eq. 1),
+//     with the sum over D .* S taken in the epilogue.
+// One CTA owns a 256 x 256 output tile as two 128 x 256 fp32 accumulators filling all 512
+// TMEM columns.  Warp 0 feeds the ring with TMA, one thread of warp 1 issues the MMAs, warps
+// 2..5 drain the accumulators.  All CTAs sweep the reduction dimension from the start at the
+// same rate, so the operand window they share stays resident in L2.
+#include <cuda_bf16.h>
+
+#include "umma.cuh"
+
+namespace adadim {
+
+// ---------------------------------------------------------------------------------------------
+// host: tensor maps
+// ---------------------------------------------------------------------------------------------
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    if (q != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+}  // namespace
+
+int make_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
+                   uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return ADADIM_ERR_CUDA;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// device
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+enum class Mode { kHessian, kScore };
+
+struct TcParams {
+  int num_tiles;            // output tiles (256 x 256) to process
+  int num_k;                // 64-deep reduction steps per tile
+  int* status_dev;
+  // Hessian
+  float* H;
+  int64_t in;               // H is [in][in]; also the column count of D
+  // Score
+  const __nv_bfloat16* D;   // [m_total][in]
+  int64_t m_total;
+  int tiles_n;              // column tiles of S
+  double* partial;          // [num_tiles][2 halves][4 warps]
+};
+
+constexpr int kKT = 64;                       // reduction depth of one ring stage
+constexpr int kTcThreads = 192;
+constexpr uint32_t kOperandBytes = 256 * kKT * 2;   // one 256-wide bf16 operand slab per stage
+
+template <Mode MODE> struct TcCfg;
+template <> struct TcCfg<Mode::kHessian> { static constexpr int NB = 1, STAGES = 3; static constexpr bool MN = true; };
+template <> struct TcCfg<Mode::kScore>   { static constexpr int NB = 2, STAGES = 2; static constexpr bool MN = false; };
+
+template <Mode MODE>
+constexpr size_t tc_smem_bytes() {
+  return static_cast<size_t>(TcCfg<MODE>::STAGES) * (1 + TcCfg<MODE>::NB) * kOperandBytes + 1024 + 256;
+}
+
+__device__ __forceinline__ void tri_coords(int t, int& rb, int& cb) {
+  int r = static_cast<int>((sqrt(8.0 * t + 1.0) - 1.0) * 0.5);
+  while (r * (r + 1) / 2 > t) --r;
+  while ((r + 1) * (r + 2) / 2 <= t) ++r;
+  rb = r;
+  cb = t - r * (r + 1) / 2;
+}
+
+template <Mode MODE>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+          const __grid_constant__ CUtensorMap tmB1, const TcParams p) {
+  using Cfg = TcCfg<MODE>;
+  constexpr int NB = Cfg::NB, STAGES = Cfg::STAGES;
+  constexpr uint32_t STAGE_BYTES = (1 + NB) * kOperandBytes;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* full = bars;                   // [STAGES] TMA -> MMA
+  uint64_t* empty = bars + STAGES;         // [STAGES] MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;  // MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 1;      // epilogue -> MMA
+  uint64_t* drain = acc_full + 2;          // used only when a wait ran out
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 3);
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    ptx::mbar_init(acc_full, 1);
+    ptx::mbar_init(acc_empty, 4);
+    ptx::mbar_init(drain, 1);
+    *dead = 0;
+    ptx::fence_mbar_init();
+    ptx::tma_prefetch_desc(&tmA);
+    ptx::tma_prefetch_desc(&tmB0);
+    if (NB == 2) ptx::tma_prefetch_desc(&tmB1);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int last_phase[STAGES];
+      for (int s = 0; s < STAGES; ++s) last_phase[s] = -1;
+      for (int t = blockIdx.x; t < p.num_tiles && !*dead; t += gridDim.x) {
+        int rb, cb;
+        if (MODE == Mode::kHessian) tri_coords(t, rb, cb); else { rb = t / p.tiles_n; cb = t % p.tiles_n; }
+        const bool shared_operand = (MODE == Mode::kHessian) && rb == cb;   // B is A on the diagonal
+        for (int k = 0; k < p.num_k; ++k) {
+          if (!ptx::mbar_wait(&empty[stage], phase ^ 1u, dead, p.status_dev)) break;
+          uint8_t* a_dst = smem + stage * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + kOperandBytes;
+          ptx::mbar_arrive_expect_tx(&full[stage], shared_operand ? kOperandBytes : STAGE_BYTES);
+          last_phase[stage] = static_cast<int>(phase);
+          if (MODE == Mode::kHessian) {
+            // X is [tokens][in]: boxes of 64 channels x 64 tokens, channels contiguous (MN-major)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              ptx::tma_load_2d(a_dst + j * (kKT * 128), &tmA, rb * 256 + j * 64, k * kKT, &full[stage]);
+            if (!shared_operand) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                ptx::tma_load_2d(b_dst + j * (kKT * 128), &tmB0, cb * 256 + j * 64, k * kKT, &full[stage]);
+            }
+          } else {
+            // D is [rows][in] and H is [in][in]: boxes of 64 reduction elements x 256 rows (K-major)
+            ptx::tma_load_2d(a_dst, &tmA, k * kKT, rb * 256, &full[stage]);
+            ptx::tma_load_2d(b_dst, &tmB0, k * kKT, cb * 256, &full[stage]);
+            ptx::tma_load_2d(b_dst + kOperandBytes, &tmB1, k * kKT, cb * 256, &full[stage]);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (*dead) {
+        // a wait ran out somewhere: let the copies already issued land before shared memory goes away
+        for (int s = 0; s < STAGES; ++s) {
+          if (last_phase[s] < 0) continue;
+          const long long t0 = clock64();
+          while (!ptx::mbar_try_wait(&full[s], static_cast<uint32_t>(last_phase[s])) && clock64() - t0 < ptx::kWaitLimit) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16(128, 256, Cfg::MN, Cfg::MN);
+      // MN-major: 64-channel blocks are kKT*128 bytes apart (LBO), 8-token groups 1024 bytes (SBO).
+      // K-major: 8-row groups are 1024 bytes apart (SBO); LBO is not used with a 128-byte swizzle.
+      constexpr uint64_t desc = Cfg::MN ? ptx::smem_desc_sw128(kKT * 128, 1024) : ptx::smem_desc_sw128(16, 1024);
+      constexpr uint32_t a_half = Cfg::MN ? 2 * kKT * 128 : 128 * 128;   // bytes between the two 128-row halves of A
+      constexpr uint32_t k16_step = Cfg::MN ? 16 * 128 : 32;             // bytes per 16 reduction elements
+      int stage = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      for (int t = blockIdx.x; t < p.num_tiles && !*dead; t += gridDim.x) {
+        int rb, cb;
+        if (MODE == Mode::kHessian) tri_coords(t, rb, cb); else { rb = t / p.tiles_n; cb = t % p.tiles_n; }
+        const bool shared_operand = (MODE == Mode::kHessian) && rb == cb;
+        if (!ptx::mbar_wait(acc_empty, acc_phase ^ 1u, dead, p.status_dev)) break;
+        ptx::tc_fence_after_sync();
+        bool ok = true;
+        for (int k = 0; k < p.num_k; ++k) {
+          if (!ptx::mbar_wait(&full[stage], phase, dead, p.status_dev)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t a_addr = ptx::smem_addr(smem + stage * STAGE_BYTES);
+          const uint32_t b_addr = shared_operand ? a_addr : a_addr + kOperandBytes;
+#pragma unroll
+          for (int k16 = 0; k16 < kKT / 16; ++k16) {
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {
+#pragma unroll
+              for (int b = 0; b < NB; ++b) {
+                ptx::mma_f16(tmem_base + a * 256,
+                             ptx::with_start(desc, a_addr + a * a_half + k16 * k16_step),
+                             ptx::with_start(desc, b_addr + b * kOperandBytes + k16 * k16_step),
+                             idesc, (k | k16 | b) != 0);
+              }
+            }
+          }
+          ptx::mma_commit(&empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::mma_commit(acc_full);
+        acc_phase ^= 1u;
+      }
+      if (*dead) {
+        ptx::mma_commit(drain);
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(drain, 0) && clock64() - t0 < ptx::kWaitLimit) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                       // TMEM lane quadrant this warp may read
+    uint32_t acc_phase = 0;
+    for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
+      int rb, cb;
+      if (MODE == Mode::kHessian) tri_coords(t, rb, cb); else { rb = t / p.tiles_n; cb = t % p.tiles_n; }
+      const bool live = ptx::mbar_wait(acc_full, acc_phase, dead, p.status_dev);
+      if (!live) break;
+      ptx::tc_fence_after_sync();
+      double part[2] = {0.0, 0.0};
+#pragma unroll 1
+      for (int a = 0; a < 2; ++a) {
+        const int64_t i = static_cast<int64_t>(rb) * 256 + a * 128 + q * 32 + lane;
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          float v[32];
+          ptx::tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * 256 + c * 32, v);
+          const int64_t j0 = static_cast<int64_t>(cb) * 256 + c * 32;
+          if (MODE == Mode::kHessian) {
+            if (i < p.in) {
+              float* hrow = p.H + i * p.in + j0;
+#pragma unroll
+              for (int k4 = 0; k4 < 8; ++k4) {
+                if (j0 + k4 * 4 < p.in) {
+                  float4 h = *reinterpret_cast<float4*>(hrow + k4 * 4);
+                  h.x += 2.0f * v[k4 * 4 + 0]; h.y += 2.0f * v[k4 * 4 + 1];
+                  h.z += 2.0f * v[k4 * 4 + 2]; h.w += 2.0f * v[k4 * 4 + 3];
+                  *reinterpret_cast<float4*>(hrow + k4 * 4) = h;
+                }
+              }
+              if (rb != cb) {                       // mirror into the upper triangle
+#pragma unroll
+                for (int k = 0; k < 32; ++k)
+                  if (j0 + k < p.in) p.H[(j0 + k) * p.in + i] += 2.0f * v[k];
+              }
+            }
+          } else {
+            if (i < p.m_total && j0 < p.in) {       // in % 64 == 0: a 32-column chunk is all in or out
+              const uint4* dp = reinterpret_cast<const uint4*>(p.D + i * p.in + j0);
+              float acc = 0.0f;
+#pragma unroll
+              for (int k8 = 0; k8 < 4; ++k8) {
+                uint4 raw = dp[k8];
+                const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                  float2 f = __bfloat1622float2(d2[m]);
+                  acc = fmaf(f.x, v[k8 * 8 + 2 * m], acc);
+                  acc = fmaf(f.y, v[k8 * 8 + 2 * m + 1], acc);
+                }
+              }
+              part[a] += static_cast<double>(acc);
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(acc_empty);
+      if (MODE == Mode::kScore) {
+        // one partial per (tile, 128-row half, warp): no cross-warp synchronisation needed
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+          double s = part[a];
+          for (int m = 16; m > 0; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
+          if (lane == 0) p.partial[(static_cast<int64_t>(t) * 2 + a) * 4 + q] = s;
+        }
+      }
+      acc_phase ^= 1u;
+    }
+  }
+
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---- fp32 activations: plain FFMA kernel (small calibration sets; keeps full fp32 products) ----
+__global__ void __launch_bounds__(256)
+hessian_f32_kernel(const float* __restrict__ X, int64_t n_tokens, int64_t in, int64_t ldx, float* __restrict__ H) {
+  // one 64 x 64 lower-triangle tile of H per CTA, 4 x 4 outputs per thread
+  __shared__ float sa[16][64 + 4];
+  __shared__ float sb[16][64 + 4];
+  int rb, cb;
+  tri_coords(blockIdx.x, rb, cb);
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  float acc[4][4] = {};
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += 16) {
+    for (int e = threadIdx.x; e < 16 * 64; e += 256) {
+      int tt = e >> 6, c = e & 63;
+      int64_t tok = t0 + tt;
+      int64_t ia = static_cast<int64_t>(rb) * 64 + c, ib = static_cast<int64_t>(cb) * 64 + c;
+      sa[tt][c] = (tok < n_tokens && ia < in) ? X[tok * ldx + ia] : 0.0f;
+      sb[tt][c] = (tok < n_tokens && ib < in) ? X[tok * ldx + ib] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int tt = 0; tt < 16; ++tt) {
+      float a[4], b[4];
+#pragma unroll
+      for (int m = 0; m < 4; ++m) { a[m] = sa[tt][ty * 4 + m]; b[m] = sb[tt][tx * 4 + m]; }
+#pragma unroll
+      for (int m = 0; m < 4; ++m)
+#pragma unroll
+        for (int n = 0; n < 4; ++n) acc[m][n] = fmaf(a[m], b[n], acc[m][n]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int m = 0; m < 4; ++m)
+#pragma unroll
+    for (int n = 0; n < 4; ++n) {
+      int64_t i = static_cast<int64_t>(rb) * 64 + ty * 4 + m, j = static_cast<int64_t>(cb) * 64 + tx * 4 + n;
+      if (i < in && j < in) {
+        if (rb != cb) {
+          H[i * in + j] += 2.0f * acc[m][n];
+          H[j * in + i] += 2.0f * acc[m][n];
+        } else {
+          H[i * in + j] += 2.0f * acc[m][n];     // the diagonal tile computes its full square
+        }
+      }
+    }
+}
+
+template <Mode MODE>
+int tc_launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const TcParams& p, cudaStream_t st) {
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    ADADIM_CUDA_TRY(cudaGetDevice(&dev));
+    ADADIM_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
+  ADADIM_CUDA_TRY(cudaFuncSetAttribute(tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(tc_smem_bytes<MODE>())));
+  int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
+  tc_kernel<MODE><<<grid, kTcThreads, tc_smem_bytes<MODE>(), st>>>(a, b0, b1, p);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+}  // namespace
+
+int hessian_bf16_launch(const void* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, int* status_dev,
+                        cudaStream_t st) {
+  CUtensorMap tm;
+  int rc = make_tmap_bf16(&tm, X, static_cast<uint64_t>(in), static_cast<uint64_t>(n_tokens),
+                          static_cast<uint64_t>(ldx) * 2, kKT);
+  if (rc != ADADIM_OK) return rc;
+  TcParams p = {};
+  const int nblk = static_cast<int>((in + 255) / 256);
+  p.num_tiles = nblk * (nblk + 1) / 2;
+  p.num_k = static_cast<int>((n_tokens + kKT - 1) / kKT);
+  p.status_dev = status_dev;
+  p.H = H;
+  p.in = in;
+  return tc_launch<Mode::kHessian>(tm, tm, tm, p, st);
+}
+
+int hessian_f32_launch(const float* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, cudaStream_t st) {
+  const int nblk = static_cast<int>((in + 63) / 64);
+  hessian_f32_kernel<<<nblk * (nblk + 1) / 2, 256, 0, st>>>(X, n_tokens, in, ldx, H);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+// S = D * (Hhi + Hlo); partial[tile][half][warp] = that warp's share of the sum of D .* S over the
+// tile's 128-row half.
+int score_gemm_launch(const __nv_bfloat16* D, int64_t m_total, int64_t in, const __nv_bfloat16* Hhi,
+                      const __nv_bfloat16* Hlo, double* partial, int* status_dev, cudaStream_t st) {
+  CUtensorMap ta, tb0, tb1;
+  int rc = make_tmap_bf16(&ta, D, static_cast<uint64_t>(in), static_cast<uint64_t>(m_total), static_cast<uint64_t>(in) * 2, 256);
+  if (rc != ADADIM_OK) return rc;
+  rc = make_tmap_bf16(&tb0, Hhi, static_cast<uint64_t>(in), static_cast<uint64_t>(in), static_cast<uint64_t>(in) * 2, 256);
+  if (rc != ADADIM_OK) return rc;
+  rc = make_tmap_bf16(&tb1, Hlo, static_cast<uint64_t>(in), static_cast<uint64_t>(in), static_cast<uint64_t>(in) * 2, 256);
+  if (rc != ADADIM_OK) return rc;
+  TcParams p = {};
+  p.tiles_n = static_cast<int>((in + 255) / 256);
+  p.num_tiles = static_cast<int>((m_total + 255) / 256) * p.tiles_n;
+  p.num_k = static_cast<int>((in + kKT - 1) / kKT);
+  p.status_dev = status_dev;
+  p.D = D;
+  p.in = in;
+  p.m_total = m_total;
+  p.partial = partial;
+  return tc_launch<Mode::kScore>(ta, tb0, tb1, p, st);
+}
+
+int score_tiles(int64_t m_total, int64_t in) {
+  return static_cast<int>((m_total + 255) / 256) * static_cast<int>((in + 255) / 256);
+}
+
+}  // namespace adadim
