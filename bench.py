@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the AdaDim layer-quantization path on B200.
+
+One step = one pass of the whole path over one layer: calibration Hessian over all tokens,
+RTN in both grouping dimensions, score + select, damped Cholesky-inverse factor, GPTQ in both
+dimensions, score + select.  Workload: the LLaMA-7B q_proj-shaped layer (W 4096 x 4096 fp16,
+X 262144 x 4096 bf16), 3-bit, group 128, seeded synthetic tensors.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line.  With N > 1 (under torchrun) every rank quantizes its own replica of the
+layer; there is no data-path collective.  `--impl reference` times the CPU oracle on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "AdaDim layer quant weights/s (RTN & GPTQ, 3b g128); % of HBM/tensor roofline"
+BITS, GROUP = 3, 128
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    def __init__(self, gpu_index: int):
+        self.gpu, self.rows, self.proc, self.thread = gpu_index, [], None, None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.rows:
+            if ts < t0 or ts > t1 + 0.1:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, f[2:]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- launch count
+def launches_per_step(out: int, inp: int) -> int:
+    """Kernels of this library launched by one step (mirrors the host-side launch logic)."""
+    nb = inp // 64
+    levels = 0
+    s = 64
+    while s < inp:
+        levels += 1
+        s *= 2
+    factor = 2 + nb + 2 * (nb - 1) + 1 + 2 * levels + 1
+    blocks = inp // 128
+    gptq = factor + 1 + blocks + (blocks - 1) + 1
+    hessian = 2 if inp > 256 else 1
+    rtn = 1
+    score = 2 + 1 + 1 + 1
+    return hessian + rtn + score + gptq + score
+
+
+# --------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2309_15531_b200 import binding as B
+    from paper_2309_15531_b200 import inputs as I
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = I.workload_qproj()
+    wspec, xspec = wl["layers"]["q_proj"]
+    out, inp, ntok = wspec.out, wspec.inp, xspec.n_tokens
+    W = I.make_weight(wspec, dev)
+    X = I.make_calib(xspec, dev)
+    H = torch.zeros(inp, inp, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws_g = torch.empty(B.workspace_bytes(B.WS_GPTQ, out, inp), dtype=torch.uint8, device=dev)
+    ws_s = torch.empty(B.workspace_bytes(B.WS_SCORE, out, inp), dtype=torch.uint8, device=dev)
+    ws_f = torch.empty(B.workspace_bytes(B.WS_FACTOR, 0, inp), dtype=torch.uint8, device=dev)
+    r_oc, r_ic = B.QTensor(out, inp, BITS, GROUP, B.DIM_OC, dev), B.QTensor(out, inp, BITS, GROUP, B.DIM_IC, dev)
+    g_oc, g_ic = B.QTensor(out, inp, BITS, GROUP, B.DIM_OC, dev), B.QTensor(out, inp, BITS, GROUP, B.DIM_IC, dev)
+    err_r = torch.zeros(2, dtype=torch.float64, device=dev)
+    err_g = torch.zeros(2, dtype=torch.float64, device=dev)
+    ch_r = torch.zeros(1, dtype=torch.int32, device=dev)
+    ch_g = torch.zeros(1, dtype=torch.int32, device=dev)
+    loss = torch.zeros(2, dtype=torch.float64, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)       # > 126 MB L2
+
+    stages = ["hessian", "rtn", "score_rtn", "factor", "gptq", "score_gptq"]
+
+    def one_step(Wd, Xd, ev=None):
+        def mark(i):
+            if ev is not None:
+                ev[i].record()
+        H.zero_()
+        mark(0)
+        B.hessian_accumulate(Xd, H, st)
+        mark(1)
+        B.quantize_rtn(Wd, BITS, GROUP, B.DIM_BOTH, r_oc, r_ic)
+        mark(2)
+        B.score_select(Wd, H, BITS, GROUP, r_oc, r_ic, err_r, ch_r, st, ws_s)
+        mark(3)
+        U = B.cholesky_inverse_factor(H, 0.01, st, ws_f)
+        mark(4)
+        B.quantize_gptq(Wd, H, BITS, GROUP, B.DIM_BOTH, 0.01, U, g_oc, g_ic, loss, st, ws_g)
+        mark(5)
+        B.score_select(Wd, H, BITS, GROUP, g_oc, g_ic, err_g, ch_g, st, ws_s)
+        mark(6)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step(W, X)
+    barrier()
+    assert int(st.item()) == 0, f"device status {int(st.item())}"
+
+    # ---- device-resident timing ------------------------------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
+    barrier()
+    t_wall0 = time.time()
+    for k in range(args.steps):
+        flush.fill_(k & 0xFF)                      # evict W / H / outputs from L2 between steps
+        one_step(W, X, evs[k])
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    step_ms = [evs[k][0].elapsed_time(evs[k][6]) for k in range(args.steps)]
+    stage_ms = {s: sum(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) / args.steps
+                for i, s in enumerate(stages)}
+    total_ms = sum(step_ms)
+    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    weights = out * inp
+    value = world * weights / (ms_per_step * 1e-3)
+
+    # ---- end to end: host buffers in, results out --------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        Wh = W.cpu().pin_memory()
+        Xh = X.cpu().pin_memory()
+        outs = [r_oc, r_ic, g_oc, g_ic]
+        host_out = [(torch.empty_like(q.codes, device="cpu").pin_memory(),
+                     torch.empty_like(q.scales, device="cpu").pin_memory(),
+                     torch.empty_like(q.zeros, device="cpu").pin_memory()) for q in outs]
+        host_err = torch.empty(4, dtype=torch.float64).pin_memory()
+        host_ch = torch.empty(2, dtype=torch.int32).pin_memory()
+        Wd = torch.empty_like(W)
+        Xd = X                                          # reuse the device buffer: it is overwritten by the copy
+
+        def e2e_step():
+            Wd.copy_(Wh, non_blocking=True)
+            Xd.copy_(Xh, non_blocking=True)
+            one_step(Wd, Xd)
+            for q, (c, s, z) in zip(outs, host_out):
+                c.copy_(q.codes, non_blocking=True)
+                s.copy_(q.scales, non_blocking=True)
+                z.copy_(q.zeros, non_blocking=True)
+            host_err[:2].copy_(err_r, non_blocking=True)
+            host_err[2:].copy_(err_g, non_blocking=True)
+            host_ch[:1].copy_(ch_r, non_blocking=True)
+            host_ch[1:].copy_(ch_g, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        n_e2e = max(1, min(args.steps, 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        et = torch.tensor([e0.elapsed_time(e1) / n_e2e], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(et, op=dist.ReduceOp.MAX)
+        h2d = Wh.numel() * Wh.element_size() + Xh.numel() * Xh.element_size()
+        d2h = sum(t.numel() * t.element_size() for trip in host_out for t in trip) + 4 * 8 + 2 * 4
+        e2e = {"value": world * weights / (float(et.item()) * 1e-3), "unit": "weights/s", "ms_per_step": float(et.item()),
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel ---------------------------------------------------------
+    peaks = _peaks()
+    dominant = max(stage_ms, key=stage_ms.get)
+    tile = 256
+    hess_flops = ntok * inp * (inp + tile)              # lower-triangle tiles of the symmetric product
+    rtn_bytes = weights * (2 + 2 * (BITS / 8 + 4 / GROUP))
+    score_flops = 2 * (2 * out) * inp * inp             # both dims stacked (algorithmic: one pass over H)
+    factor_flops = 2 * inp ** 3 / 3                     # Cholesky + triangular inverse
+    gptq_flops = 2 * (out * inp * inp)                  # trailing + in-block updates, both dims
+    roof_all = {
+        "hessian": {"bound": "tensor", "achieved": hess_flops / (stage_ms["hessian"] * 1e-3) / 1e12,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"},
+        "rtn": {"bound": "hbm", "achieved": rtn_bytes / (stage_ms["rtn"] * 1e-3) / 1e9,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s"},
+        "score_rtn": {"bound": "tensor", "achieved": score_flops / (stage_ms["score_rtn"] * 1e-3) / 1e12,
+                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"},
+    }
+    for v in roof_all.values():
+        v["frac"] = v["achieved"] / v["peak"]
+    if dominant in roof_all:
+        roofline = dict(roof_all[dominant])
+    elif dominant == "factor":
+        # fp64 FMA on the CUDA cores: 148 SMs x 64 FMA/clk x 2 flop at the sampled clock
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        peak = 148 * 64 * 2 * mhz * 1e6 / 1e12
+        ach = factor_flops / (stage_ms["factor"] * 1e-3) / 1e12
+        roofline = {"bound": "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak}
+    else:
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        peak = 148 * 128 * 2 * mhz * 1e6 / 1e12          # fp32 FMA on the CUDA cores
+        ach = gptq_flops / (stage_ms[dominant] * 1e-3) / 1e12
+        roofline = {"bound": "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak}
+    roofline["kernel"] = dominant
+    roofline["peak_source"] = peaks["source"] if roofline["bound"] != "alu" else "derived from unit counts and sampled clock"
+    roofline["traffic"] = None
+
+    cpu = cpu_baseline(sample_only=True)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "llama7b_q_proj W[4096,4096] fp16, X[262144,4096] bf16, 3-bit g128, "
+                               "Hessian + RTN both dims + score + factor + GPTQ both dims + score",
+                   "l2": "flushed between steps by writing a 256 MiB buffer; X (2.1 GB) exceeds L2",
+                   "replicas": world},
+        "stages_ms": stage_ms,
+        "stage_weights_per_s": {s: weights / (t * 1e-3) for s, t in stage_ms.items()},
+        "rooflines": roof_all, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": launches_per_step(out, inp) * args.steps,
+        "chosen": {"rtn": B.DIM_NAMES[int(ch_r.item())], "gptq": B.DIM_NAMES[int(ch_g.item())]},
+        "errors": {"rtn": err_r.tolist(), "gptq": err_g.tolist()},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def cpu_baseline(sample_only: bool = False):
+    """Times the oracle, as it stands, on a bounded sample of the same workload and scales each
+    stage to the full layer.  Returns the cpu_baseline object."""
+    import numpy as np
+    import torch
+    from oracle import adadim_oracle as O
+    from paper_2309_15531_b200 import inputs as I
+
+    wl = I.workload_qproj(n_tokens=1024)
+    wspec, xspec = wl["layers"]["q_proj"]
+    out, inp, full_tokens = wspec.out, wspec.inp, 128 * 2048
+    W = I.make_weight(wspec, "cpu").float().numpy()
+    X = I.make_calib(xspec, "cpu").float().numpy()
+    slab = 128
+    t = {}
+    t0 = time.time(); H = O.hessian(X); t["hessian"] = (time.time() - t0) * (full_tokens / xspec.n_tokens)
+    t0 = time.time()
+    r = {d: O.quantize_rtn(W, BITS, GROUP, d) for d in ("oc", "ic")}
+    t["rtn"] = time.time() - t0
+    t0 = time.time()
+    for d in ("oc", "ic"):
+        O.recon_error_trace(W[:512], r[d]["Q"][:512], H)
+    t["score"] = (time.time() - t0) * (out / 512) * 2           # scored twice per step (RTN and GPTQ outputs)
+    t0 = time.time(); Hd, dead = O.damped_hessian(H, 0.01); U = O.cholesky_inverse_factor(Hd); t["factor"] = time.time() - t0
+    t0 = time.time()
+    for d in ("oc", "ic"):
+        O.quantize_gptq(W[:slab], H, BITS, GROUP, d, 0.01, U=U, dead=dead)
+    t["gptq"] = (time.time() - t0) * (out / slab)
+    total = sum(t.values())
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    return {"value": out * inp / total, "unit": "weights/s", "cores": min(cores, torch.get_num_threads() or cores),
+            "kind": "oracle",
+            "sample": "Hessian on 1024 of 262144 tokens, RTN on the full W, scorer on 512 of 4096 rows, "
+                      "factor in full, GPTQ on one 128-row slab of 32; each stage scaled linearly to the full layer",
+            "stage_seconds_scaled": t}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(max(1, min(args.warmup, 1))):
+        cpu_baseline()
+    t_all = 0.0
+    last = None
+    n = max(1, min(args.steps, 3))
+    for _ in range(n):
+        last = cpu_baseline()
+        vals.append(last["value"])
+    value = sum(vals) / len(vals)
+    last["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": args.gpus,
+            "steps": n, "warmup": 1, "ms_per_step": 4096 * 4096 / value * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "llama7b_q_proj W[4096,4096] fp16, X[262144,4096] bf16, 3-bit g128 (CPU oracle, "
+                                   "bounded sample scaled to the full layer)"},
+            "cpu_baseline": last,
+            "e2e": {"value": value, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

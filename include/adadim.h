@@ -77,8 +77,9 @@ typedef struct {
  * Hessian GPTQ uses is "formed by activations"; Section 2.2).
  *   X        [n_tokens][in], xdtype ADADIM_BF16 (tcgen05 tensor-core path) or ADADIM_F32.
  *            ldx in elements; X and ldx*sizeof(elem) must be 16-byte aligned.
- *   H        [in][in] fp32, in/out: the caller zeroes it before the first chunk.  Both
- *            triangles are updated.  in must be a multiple of 8.
+ *   H        [in][in] fp32, in/out, symmetric on entry: the caller zeroes it before the first
+ *            chunk and passes it back unchanged for the next ones.  Both triangles are valid
+ *            on return.  in must be a multiple of 8.
  *   n_seen   host pointer, in/out, may be NULL: incremented by n_tokens.
  *   status_dev  device int, may be NULL.
  *   workspace   unused by the current kernels (adadim_workspace_bytes(ADADIM_WS_HESSIAN,..)
@@ -127,7 +128,8 @@ ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, float 
  * (already compensated) weights with the formula of adadim_quantize_rtn: per-OC at each
  * group's first column, from that group's columns; per-IC at every column, from its g-row
  * groups.  Weights of dead columns are treated as 0.
- *   H          [in][in] fp32, used when U == NULL (the factor is then computed into workspace).
+ *   H          [in][in] fp32, required: its diagonal marks the dead columns, and when U == NULL
+ *              the factor is computed from it into workspace.
  *   U          optional precomputed adadim_cholesky_inverse_factor of the same H, or NULL.
  *   blocksize  128.  group must divide 128.  in % 128 == 0, out % 128 == 0.
  *   gptq_loss  optional device double[2] (OC, IC): 1/2 * sum of e^2.

@@ -56,7 +56,7 @@ def group_params(lo, hi, bits):
         bad = (s == 0) | ~np.isfinite(s)
         s = np.where(bad, F32(1), s).astype(F32)
         z = np.rint(((-lo) / s).astype(F32)).astype(F32)
-        z = np.clip(z, F32(0), maxq).astype(F32)
+        z = (np.clip(z, F32(0), maxq) + F32(0)).astype(F32)      # an integer 0..maxq: never -0.0
         z = np.where(bad, F32(0), z).astype(F32)
     return s, z, bad
 

@@ -66,7 +66,7 @@ __device__ __forceinline__ GroupParams group_params(float lo, float hi, float ma
     g.s = 1.0f; g.z = 0.0f; g.rcp = 0.0f;
   } else {
     g.s = s;
-    g.z = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), maxq);
+    g.z = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), maxq) + 0.0f;   // + 0: never store -0
     g.rcp = __frcp_rn(s);
   }
   return g;

@@ -104,7 +104,7 @@ def test_one_signed_and_degenerate_groups():
     # all-positive group: the range is extended down to zero, zero point 0
     W = np.linspace(0.5, 1.2, 128, dtype=np.float32)[None, :]
     r = O.quantize_rtn(W, 3, 128, "oc")
-    assert r["zeros"][0, 0] == 0
+    assert r["zeros"][0, 0] == 0 and r["zeros"].view(np.uint16)[0, 0] == 0      # +0, never -0
     assert abs(float(r["scales"][0, 0]) * 7 - 1.2) < 1.2 * 2.0 ** -10
     # all-negative group: zero point is maxq
     r = O.quantize_rtn(-W, 3, 128, "oc")
