@@ -11,8 +11,9 @@
  * Conventions that hold for every entry point
  *   - All matrices are row-major.  W[o,i] is at W + o*ldw + i; X[t,i] (token t) at X + t*ldx + i.
  *   - Unless an argument is marked "host", every pointer is a DEVICE pointer owned by the
- *     caller.  The library allocates no device memory and keeps no state between calls;
- *     inputs are never modified.
+ *     caller.  The library allocates no device memory and keeps no state between calls
+ *     (the one exception, a built-in scratch array, is described at
+ *     adadim_score_select_static); inputs are never modified.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *     stream).  No entry point synchronizes; results are valid once the stream has run.
  *   - The return value is an adadim_status.  Argument errors are found on the host before
@@ -157,6 +158,39 @@ ADADIM_API int adadim_score_select(const void* W, int wdtype, int64_t out, int64
                         const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                         double* err, int* chosen, int* status_dev,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * adadim_score_select without a workspace argument, for callers that cannot allocate device
+ * memory (the paper has no counterpart: this is a convenience of this library).
+ *
+ * Who needs it: code that may not call cudaMalloc - a component running inside a process
+ * whose device memory is already fully committed (an inference server that gave every free
+ * byte to its cache), a plugin that receives tensors but no allocator, or a latency-critical
+ * path that cannot accept the device-wide synchronisation an allocation may imply.  Such a
+ * caller still passes all inputs and outputs; only the scratch comes from the library: a
+ * fixed array of ADADIM_STATIC_SCRATCH_BYTES (16 MiB) in the library's device image, present
+ * on every GPU that loads the library for as long as the process lives.
+ *
+ *   Limit      adadim_workspace_bytes(ADADIM_WS_SCORE, out, in, ..) must not exceed
+ *              ADADIM_STATIC_SCRATCH_BYTES (for example out = in = 1024 fits, out = in = 2048
+ *              does not); larger layers are refused with ADADIM_ERR_WORKSPACE and nothing is
+ *              launched.
+ *   First call The first call on each device looks up the array's device address; make that
+ *              first call on a device outside any stream capture.
+ *   Sharing    All calls on a device use the same array.  It keeps the previous call's
+ *              contents, which no call reads (each call rewrites what it uses).  Two calls
+ *              whose kernels can overlap on the GPU - different streams, or different host
+ *              threads using different streams - race on it and give wrong results: keep
+ *              calls on one device ordered on a single stream, or otherwise serialized.
+ *   No cudaMalloc, cudaFree or other allocating call is made.  Arguments, results, status
+ *   codes and numerical behaviour are otherwise those of adadim_score_select.
+ */
+#define ADADIM_STATIC_SCRATCH_BYTES (16u << 20)
+ADADIM_API int adadim_score_select_static(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
+                                          const float* H, int bits, int group,
+                                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+                                          double* err, int* chosen, int* status_dev, void* cuda_stream);
+ADADIM_API size_t adadim_static_scratch_bytes(void);
 
 /* Helpers. */
 ADADIM_API size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int group);

@@ -60,6 +60,10 @@ def lib():
         L.adadim_score_select.restype = C.c_int
         L.adadim_score_select.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, qp, qp, vp, vp, vp, vp,
                                           sz, vp]
+        L.adadim_score_select_static.restype = C.c_int
+        L.adadim_score_select_static.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, qp, qp, vp, vp,
+                                                 vp, vp]
+        L.adadim_static_scratch_bytes.restype = sz
         L.adadim_unpack_codes.restype = C.c_int
         L.adadim_unpack_codes.argtypes = [vp, i64, i64, C.c_int, vp, vp]
         _lib = L
@@ -202,3 +206,26 @@ def score_select(W: torch.Tensor, H: torch.Tensor, bits: int, group: int,
                                    workspace.data_ptr(), workspace.numel(), _stream())
     _check(rc, "adadim_score_select")
     return err, chosen
+
+
+def static_scratch_bytes() -> int:
+    return int(lib().adadim_static_scratch_bytes())
+
+
+def score_select_static(W: torch.Tensor, H: torch.Tensor, bits: int, group: int,
+                        q_oc: Optional[QTensor], q_ic: Optional[QTensor],
+                        err: torch.Tensor, chosen: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
+    """score_select on the library's built-in scratch array, for callers that cannot allocate
+    device memory.  The caller passes every buffer, outputs included (err float64[2], chosen
+    int32[1]); this wrapper creates no tensor.  Layers whose scoring workspace exceeds
+    static_scratch_bytes() raise AdadimError(status 6).  Calls on one device must not overlap
+    on the GPU: they share the array."""
+    out, inp = W.shape
+    coc = q_oc.c() if q_oc is not None else None
+    cic = q_ic.c() if q_ic is not None else None
+    rc = lib().adadim_score_select_static(W.data_ptr(), _DT[W.dtype], out, inp, W.stride(0), H.data_ptr(), bits, group,
+                                          C.byref(coc) if coc is not None else None,
+                                          C.byref(cic) if cic is not None else None,
+                                          err.data_ptr(), chosen.data_ptr(),
+                                          status.data_ptr() if status is not None else None, _stream())
+    _check(rc, "adadim_score_select_static")
