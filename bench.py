@@ -89,18 +89,25 @@ class ClockSampler:
 def launches_per_step(out: int, inp: int) -> int:
     """Kernels of this library launched by one step (mirrors the host-side launch logic)."""
     nb = inp // 64
-    levels = 0
-    s = 64
+    factor = 2                                           # damping, build
+    for g0 in range(0, nb, 4):
+        g1 = min(g0 + 4, nb)
+        for k in range(g0, g1):
+            below, inner = nb - k - 1, g1 - k - 1
+            factor += 1 + (1 if below > 0 else 0) + (1 if below > 0 and inner > 0 else 0)
+        factor += 1 if g1 * 64 < inp else 0              # rank-256 update
+    factor += 1 + (2 if inp > 64 else 0)                 # seed, 64-level merges
+    s = 128
     while s < inp:
-        levels += 1
+        factor += 2
         s *= 2
-    factor = 2 + nb + 2 * (nb - 1) + 1 + 2 * levels + 1
+    factor += 1                                          # emit
     blocks = inp // 128
-    gptq = factor + 1 + blocks + (blocks - 1) + 1
+    gptq = 1 + 1 + blocks + (blocks - 1) + 1           # init, U slicing, block kernels, trailing kernels, loss
     hessian = 2 if inp > 256 else 1
     rtn = 1
     score = 2 + 1 + 1 + 1
-    return hessian + rtn + score + gptq + score
+    return hessian + rtn + score + factor + gptq + score
 
 
 # --------------------------------------------------------------------------- our arm
@@ -278,7 +285,7 @@ def run_ours(args):
     roofline["peak_source"] = peaks["source"] if roofline["bound"] != "alu" else "derived from unit counts and sampled clock"
     roofline["traffic"] = None
 
-    cpu = cpu_baseline(sample_only=True)
+    cpu = None if args.no_cpu_baseline else cpu_baseline()
 
     line = {
         "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
@@ -301,7 +308,7 @@ def run_ours(args):
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
-def cpu_baseline(sample_only: bool = False):
+def cpu_baseline():
     """Times the oracle, as it stands, on a bounded sample of the same workload and scales each
     stage to the full layer.  Returns the cpu_baseline object."""
     import numpy as np
@@ -370,6 +377,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -8,17 +8,25 @@
 // binary64 on the CUDA cores (the factor decides GPTQ's rounding, so it is kept well inside
 // the fp32 precision of U); U is rounded to fp32 on output.
 //
-//   factorization : right-looking, 64-column panels (diagonal block on one CTA, then a panel
-//                   multiply by the inverted diagonal block, then the trailing update)
+//   factorization : 64-column panels (diagonal block on one CTA, then the panel below it
+//                   multiplied by the inverted diagonal block).  Panels are grouped four at a
+//                   time: inside a group only the group's own columns are updated after each
+//                   panel; the rest of the matrix gets one rank-256 update per group, on
+//                   128 x 128 tiles (high arithmetic intensity).
 //   inverse       : recursive doubling.  inv([[A,0],[C,B]]) = [[A^-1,0],[-B^-1 C A^-1,B^-1]]:
 //                   level by level, adjacent inverted diagonal blocks are merged with two
 //                   batched triangular-aware matrix products, log2(n/64) levels in all.
+// The strict upper triangle of the work matrix is kept at zero outside 64-blocks on the
+// diagonal, so whole diagonal tiles can be used as triangular operands.
 #include "common.cuh"
 
 namespace adadim {
 namespace {
 
-constexpr int kNB = 64;     // panel width and tile edge
+constexpr int kNB = 64;     // panel width and small tile edge
+constexpr int kGroup = 4;   // panels per rank-256 update
+
+__host__ __device__ __forceinline__ int64_t mn64(int64_t a, int64_t b) { return a < b ? a : b; }
 
 // ---- 64 x 64 output tile product, 256 threads, 4 x 4 outputs per thread --------------------
 // acc += A[64 x K] * B, A row-major with leading dimension lda;
@@ -65,6 +73,91 @@ __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64
   __shared__ double sa[16][kNB + 2];   \
   __shared__ double sb[16][kNB + 2];
 
+// ---- 128 x 128 output tile product, 256 threads, 8 x 8 outputs per thread ------------------
+// Output rows of a thread: ty*4 + {0..3} and 64 + ty*4 + {0..3}; columns likewise with tx.
+// Rows >= a_rows of A and columns >= b_cols of B are not read (treated as zero); both limits
+// are 64 or 128.  K is a multiple of 8.  Shared-memory slabs are double-buffered and the next
+// slab is fetched into registers while the current one is multiplied.
+constexpr int kT = 128, kBK = 8, kLd = kT + 4;
+struct Tile128Smem {
+  double a[2][kBK][kLd];
+  double b[2][kBK][kLd];
+};
+
+template <bool B_T>
+__device__ __forceinline__ void product128(const double* __restrict__ A, int64_t lda, int a_rows,
+                                           const double* __restrict__ B, int64_t ldb, int b_cols, int K,
+                                           double (&acc)[8][8], Tile128Smem& sm) {
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int ar = tid >> 1, akq = (tid & 1) * 4;                 // A loader: row, first k of four
+  const int bkk = tid >> 5, bnq = (tid & 31) * 4;               // B loader (not transposed): k row, first col
+  const bool a_ok = ar < a_rows;
+  const bool b_ok = B_T ? (ar < b_cols) : (bnq < b_cols);
+  const double* ap = A + static_cast<int64_t>(ar) * lda + akq;
+  const double* bp = B_T ? B + static_cast<int64_t>(ar) * ldb + akq : B + static_cast<int64_t>(bkk) * ldb + bnq;
+  const int64_t bstep = B_T ? kBK : static_cast<int64_t>(kBK) * ldb;
+  double2 ra0, ra1, rb0, rb1;
+  const double2 zero2 = make_double2(0.0, 0.0);
+
+  auto fetch = [&](int k0) {
+    if (a_ok) { const double2* s = reinterpret_cast<const double2*>(ap + k0); ra0 = s[0]; ra1 = s[1]; }
+    else { ra0 = zero2; ra1 = zero2; }
+    if (b_ok) { const double2* s = reinterpret_cast<const double2*>(bp + (k0 / kBK) * bstep); rb0 = s[0]; rb1 = s[1]; }
+    else { rb0 = zero2; rb1 = zero2; }
+  };
+  auto stash = [&](int buf) {
+    sm.a[buf][akq + 0][ar] = ra0.x; sm.a[buf][akq + 1][ar] = ra0.y;
+    sm.a[buf][akq + 2][ar] = ra1.x; sm.a[buf][akq + 3][ar] = ra1.y;
+    if (B_T) {
+      sm.b[buf][akq + 0][ar] = rb0.x; sm.b[buf][akq + 1][ar] = rb0.y;
+      sm.b[buf][akq + 2][ar] = rb1.x; sm.b[buf][akq + 3][ar] = rb1.y;
+    } else {
+      *reinterpret_cast<double2*>(&sm.b[buf][bkk][bnq]) = rb0;
+      *reinterpret_cast<double2*>(&sm.b[buf][bkk][bnq + 2]) = rb1;
+    }
+  };
+
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < K; k0 += kBK) {
+    const bool more = k0 + kBK < K;
+    if (more) fetch(k0 + kBK);
+#pragma unroll
+    for (int kk = 0; kk < kBK; ++kk) {
+      double a[8], b[8];
+      *reinterpret_cast<double2*>(a + 0) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4]);
+      *reinterpret_cast<double2*>(a + 2) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4 + 2]);
+      *reinterpret_cast<double2*>(a + 4) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4]);
+      *reinterpret_cast<double2*>(a + 6) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4 + 2]);
+      *reinterpret_cast<double2*>(b + 0) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][tx * 4]);
+      *reinterpret_cast<double2*>(b + 2) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][tx * 4 + 2]);
+      *reinterpret_cast<double2*>(b + 4) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][64 + tx * 4]);
+      *reinterpret_cast<double2*>(b + 6) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][64 + tx * 4 + 2]);
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+#pragma unroll
+        for (int n = 0; n < 8; ++n) acc[m][n] = fma(a[m], b[n], acc[m][n]);
+    }
+    if (more) stash(buf ^ 1);
+    __syncthreads();
+    buf ^= 1;
+  }
+}
+
+// Applies f(row, col4, values of 4 consecutive columns) to a thread's 8 x 8 outputs.
+template <typename F>
+__device__ __forceinline__ void for_each_quad(double (&acc)[8][8], F f) {
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int m = 0; m < 8; ++m) {
+    const int r = (m < 4 ? 0 : 64) + ty * 4 + (m & 3);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) f(r, h * 64 + tx * 4, &acc[m][h * 4]);
+  }
+}
+
 // ---- set-up --------------------------------------------------------------------------------
 // stats[0] = lambda = percdamp * mean_i diag(H) after the dead-column fix (fixed summation order).
 __global__ void __launch_bounds__(256)
@@ -84,60 +177,85 @@ damp_kernel(const float* __restrict__ H, int64_t n, double percdamp, double* sta
   if (threadIdx.x == 0) stats[0] = percdamp * red[0] / static_cast<double>(n);
 }
 
-// A[r][c] = Hd[n-1-r][n-1-c]
+// A[r][c] = Hd[n-1-r][n-1-c] on and below the diagonal, 0 above it
 __global__ void __launch_bounds__(256)
 build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ stats, double* __restrict__ A) {
   int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
   if (e >= n * n) return;
   int64_t r = e / n, c = e % n;
-  int64_t i = n - 1 - r, j = n - 1 - c;
-  double v = static_cast<double>(H[i * n + j]);
-  if (i == j) {
-    if (v == 0.0) v = 1.0;
-    v += stats[0];
+  double v = 0.0;
+  if (r >= c) {
+    int64_t i = n - 1 - r, j = n - 1 - c;
+    v = static_cast<double>(H[i * n + j]);
+    if (i == j) {
+      if (v == 0.0) v = 1.0;
+      v += stats[0];
+    }
   }
   A[e] = v;
 }
 
 // ---- factorization -------------------------------------------------------------------------
 // Diagonal block k: in-place Cholesky of the 64 x 64 block and its triangular inverse -> dinv[k].
+// Column by column (left-looking): four threads share a row's dot product; the pivot's
+// reciprocal square root scales the column.  The inverse is a forward substitution with four
+// threads per column, the column's entries spread over their registers.
 __global__ void __launch_bounds__(256)
 potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv, int* status_dev) {
   __shared__ double L[kNB][kNB + 1];
+  __shared__ double col[kNB];
+  __shared__ double rdiag[kNB];          // 1 / L[j][j]
   double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
   for (int e = threadIdx.x; e < kNB * kNB; e += 256) L[e >> 6][e & 63] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
   __syncthreads();
+  const int row = threadIdx.x >> 2, q = threadIdx.x & 3;
+#pragma unroll
   for (int j = 0; j < kNB; ++j) {
-    double piv = L[j][j];
+    double s0 = 0.0, s1 = 0.0;
+#pragma unroll
+    for (int t = 0; t < (j + 3) / 4; ++t) {            // entries m = 4t + q < j of the two rows
+      const int m = 4 * t + q;
+      const double a = m < j ? L[row][m] : 0.0;
+      const double b = L[j][m];
+      if (t & 1) s1 = fma(a, b, s1); else s0 = fma(a, b, s0);
+    }
+    double sum = s0 + s1;
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+    if (q == 0 && row >= j) col[row] = L[row][j] - sum;
     __syncthreads();
+    double piv = col[j];
     if (!(piv > 0.0)) {
       if (threadIdx.x == 0) report(status_dev, ADADIM_ERR_NOT_PD);
       piv = 1.0;
     }
-    const double d = sqrt(piv);
-    if (threadIdx.x == 0) L[j][j] = d;
-    if (threadIdx.x > j && threadIdx.x < kNB) L[threadIdx.x][j] /= d;
-    __syncthreads();
-    // trailing rank-one update of the lower triangle
-    for (int e = threadIdx.x; e < kNB * kNB; e += 256) {
-      int r = e >> 6, c = e & 63;
-      if (c > j && r >= c) L[r][c] -= L[r][j] * L[c][j];
-    }
+    const double r = rsqrt(piv);
+    if (q == 0 && row >= j) L[row][j] = col[row] * r;
+    if (threadIdx.x == 0) rdiag[j] = r;
     __syncthreads();
   }
-  // X = L^-1 by forward substitution, one column per thread, the column held in registers.
-  // Entries above the diagonal come out as exact zeros (their right-hand side is zero).
-  double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
-  if (threadIdx.x < kNB) {
-    const int c = threadIdx.x;
-    double x[kNB];
+  // X = L^-1: thread (c, q) keeps X[m][c] for m = 4t + q in x[t]
+  {
+    const int c = row;
+    double x[kNB / 4];
+#pragma unroll
+    for (int t = 0; t < kNB / 4; ++t) x[t] = 0.0;
+    double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
 #pragma unroll
     for (int r = 0; r < kNB; ++r) {
-      double s = (r == c) ? 1.0 : 0.0;
+      double s0 = 0.0, s1 = 0.0;
 #pragma unroll
-      for (int m = 0; m < r; ++m) s = fma(-L[r][m], x[m], s);
-      x[r] = s / L[r][r];
-      dk[r * kNB + c] = x[r];
+      for (int t = 0; t < (r + 3) / 4; ++t) {            // entries m = 4t + q < r
+        const int m = 4 * t + q;
+        const double l = m < r ? L[r][m] : 0.0;
+        if (t & 1) s1 = fma(l, x[t], s1); else s0 = fma(l, x[t], s0);
+      }
+      double sum = s0 + s1;
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      const double xr = ((r == c ? 1.0 : 0.0) - sum) * rdiag[r];
+      if (q == (r & 3)) x[r >> 2] = xr;
+      if (q == 0) dk[r * kNB + c] = r < c ? 0.0 : xr;
     }
   }
   for (int e = threadIdx.x; e < kNB * kNB; e += 256) {
@@ -161,17 +279,14 @@ panel_kernel(double* __restrict__ A, int64_t n, int k, const double* __restrict_
     for (int c = 0; c < 4; ++c) tile[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + c] = acc[m][c];
 }
 
-// Trailing update after panel k:  A[i][j] -= L[i][k] L[j][k]^T  for k < j <= i (tiles of 64).
+// Update inside the current group of panels after panel k:  A[i][j] -= L[i][k] L[j][k]^T for the
+// column tiles j of the group that follow k and all row tiles i >= j.  blockIdx.x = i - (k+1),
+// blockIdx.y = j - (k+1).
 __global__ void __launch_bounds__(256)
-trailing_kernel(double* __restrict__ A, int64_t n, int k) {
+group_update_kernel(double* __restrict__ A, int64_t n, int k) {
   TILE_SMEM
-  // blockIdx.x enumerates the lower triangle (ti >= tj) of the trailing tile grid
-  int t = blockIdx.x;
-  int ti = static_cast<int>((sqrt(8.0 * t + 1.0) - 1.0) * 0.5);
-  while (ti * (ti + 1) / 2 > t) --ti;
-  while ((ti + 1) * (ti + 2) / 2 <= t) ++ti;
-  const int tj = t - ti * (ti + 1) / 2;
-  const int64_t ri = (static_cast<int64_t>(k) + 1 + ti) * kNB, rj = (static_cast<int64_t>(k) + 1 + tj) * kNB;
+  if (blockIdx.y > blockIdx.x) return;
+  const int64_t ri = (static_cast<int64_t>(k) + 1 + blockIdx.x) * kNB, rj = (static_cast<int64_t>(k) + 1 + blockIdx.y) * kNB;
   const int64_t ck = static_cast<int64_t>(k) * kNB;
   double acc[4][4] = {};
   tile_product<true>(A + ri * n + ck, n, A + rj * n + ck, n, kNB, acc, sa, sb);
@@ -181,6 +296,32 @@ trailing_kernel(double* __restrict__ A, int64_t n, int k) {
   for (int m = 0; m < 4; ++m)
 #pragma unroll
     for (int q = 0; q < 4; ++q) c[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + q] -= acc[m][q];
+}
+
+// Rank-`kw` update of everything right of a finished group:  for 128 x 128 tiles (ti >= tj) of
+// the region starting at row/column e:  A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T.
+// Diagonal tiles do not store their upper-right 64 x 64 quadrant (it must stay zero).
+__global__ void __launch_bounds__(256, 1)
+rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
+  __shared__ Tile128Smem sm;
+  int t = blockIdx.x;
+  int ti = static_cast<int>((sqrt(8.0 * t + 1.0) - 1.0) * 0.5);
+  while (ti * (ti + 1) / 2 > t) --ti;
+  while ((ti + 1) * (ti + 2) / 2 <= t) ++ti;
+  const int tj = t - ti * (ti + 1) / 2;
+  const int64_t ri = e + static_cast<int64_t>(ti) * kT, rj = e + static_cast<int64_t>(tj) * kT;
+  const int vr = static_cast<int>(mn64(kT, n - ri)), vc = static_cast<int>(mn64(kT, n - rj));
+  double acc[8][8] = {};
+  product128<true>(A + ri * n + j0, n, vr, A + rj * n + j0, n, vc, kw, acc, sm);
+  const bool diag = ti == tj;
+  for_each_quad(acc, [&](int r, int c4, const double* v) {
+    if (r >= vr || c4 >= vc) return;
+    if (diag && r < 64 && c4 >= 64) return;
+    double2* p = reinterpret_cast<double2*>(A + (ri + r) * n + rj + c4);
+    double2 u0 = p[0], u1 = p[1];
+    u0.x -= v[0]; u0.y -= v[1]; u1.x -= v[2]; u1.y -= v[3];
+    p[0] = u0; p[1] = u1;
+  });
 }
 
 // ---- inverse by recursive doubling -----------------------------------------------------------
@@ -195,44 +336,80 @@ seed_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ dinv) 
 
 // Level with half-size s (elements): pair p covers [p*2s, p*2s+2s); its A part is the first s
 // rows/cols (already inverted: XA), its B part the rest (XB, sB <= s rows), C the block below A.
+// T is packed pair after pair (every earlier pair has s B-rows), rows local to the B part, pitch s.
 // step 1:  T = C * XA      (T tile (r,c): reduction over XA rows m >= c only, XA is lower)
+// step 2:  C <- -XB * T    (C tile (r,c): reduction over XB columns m <= r only)
 __global__ void __launch_bounds__(256)
-merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T) {
+merge1_64_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ T) {      // s == 64
   TILE_SMEM
-  const int tiles = static_cast<int>(s / kNB);
-  const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  const int r = blockIdx.x / tiles, c = blockIdx.x % tiles;
-  if (b0 + static_cast<int64_t>(r) * kNB >= n) return;
+  const int64_t s = kNB, a0 = static_cast<int64_t>(blockIdx.x) * 2 * s, b0 = a0 + s;
+  if (b0 >= n) return;
   double acc[4][4] = {};
-  const int64_t m0 = static_cast<int64_t>(c) * kNB;
-  tile_product<false>(A + (b0 + static_cast<int64_t>(r) * kNB) * n + a0 + m0, n, A + (a0 + m0) * n + a0 + m0, n,
-                      static_cast<int>(s - m0), acc, sa, sb);
-  // T is packed pair after pair (every earlier pair has s B-rows), rows local to the B part
-  double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kNB * s + m0;
+  tile_product<false>(A + b0 * n + a0, n, A + a0 * n + a0, n, kNB, acc, sa, sb);
+  double* t = T + static_cast<int64_t>(blockIdx.x) * s * s;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
   for (int m = 0; m < 4; ++m)
 #pragma unroll
-    for (int q = 0; q < 4; ++q) t[static_cast<int64_t>(ty * 4 + m) * s + tx * 4 + q] = acc[m][q];
+    for (int q = 0; q < 4; ++q) t[(ty * 4 + m) * s + tx * 4 + q] = acc[m][q];
 }
-// step 2:  C <- -XB * T    (C tile (r,c): reduction over XB columns m <= r only)
 __global__ void __launch_bounds__(256)
-merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T) {
+merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T) {      // s == 64
   TILE_SMEM
-  const int tiles = static_cast<int>(s / kNB);
-  const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  const int r = blockIdx.x / tiles, c = blockIdx.x % tiles;
-  const int64_t row0 = b0 + static_cast<int64_t>(r) * kNB;
-  if (row0 >= n) return;
+  const int64_t s = kNB, a0 = static_cast<int64_t>(blockIdx.x) * 2 * s, b0 = a0 + s;
+  if (b0 >= n) return;
   double acc[4][4] = {};
-  tile_product<false>(A + row0 * n + b0, n, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kNB, s,
-                      (r + 1) * kNB, acc, sa, sb);
-  double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kNB;
+  tile_product<false>(A + b0 * n + b0, n, T + static_cast<int64_t>(blockIdx.x) * s * s, s, kNB, acc, sa, sb);
+  double* dst = A + b0 * n + a0;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
   for (int m = 0; m < 4; ++m)
 #pragma unroll
     for (int q = 0; q < 4; ++q) dst[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + q] = -acc[m][q];
+}
+
+__global__ void __launch_bounds__(256, 1)
+merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T) {      // s >= 128
+  __shared__ Tile128Smem sm;
+  const int tiles = static_cast<int>(s / kT);
+  const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
+  const int r = blockIdx.x / tiles, c = blockIdx.x % tiles;
+  const int64_t sB = mn64(s, n - b0);
+  if (static_cast<int64_t>(r) * kT >= sB) return;
+  const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
+  const int64_t m0 = static_cast<int64_t>(c) * kT;
+  double acc[8][8] = {};
+  product128<false>(A + (b0 + static_cast<int64_t>(r) * kT) * n + a0 + m0, n, vr, A + (a0 + m0) * n + a0 + m0, n, kT,
+                    static_cast<int>(s - m0), acc, sm);
+  double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kT * s + m0;
+  for_each_quad(acc, [&](int rr, int c4, const double* v) {
+    if (rr >= vr) return;
+    double2* p = reinterpret_cast<double2*>(t + static_cast<int64_t>(rr) * s + c4);
+    p[0] = make_double2(v[0], v[1]);
+    p[1] = make_double2(v[2], v[3]);
+  });
+}
+__global__ void __launch_bounds__(256, 1)
+merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T) {      // s >= 128
+  __shared__ Tile128Smem sm;
+  const int tiles = static_cast<int>(s / kT);
+  const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
+  const int r = blockIdx.x / tiles, c = blockIdx.x % tiles;
+  const int64_t sB = mn64(s, n - b0);
+  if (static_cast<int64_t>(r) * kT >= sB) return;
+  const int64_t row0 = b0 + static_cast<int64_t>(r) * kT;
+  const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
+  const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kT, sB));
+  double acc[8][8] = {};
+  product128<false>(A + row0 * n + b0, n, vr, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kT, s,
+                    kT, K, acc, sm);
+  double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kT;
+  for_each_quad(acc, [&](int rr, int c4, const double* v) {
+    if (rr >= vr) return;
+    double2* p = reinterpret_cast<double2*>(dst + static_cast<int64_t>(rr) * n + c4);
+    p[0] = make_double2(-v[0], -v[1]);
+    p[1] = make_double2(-v[2], -v[3]);
+  });
 }
 
 // U[i][j] = Linv[n-1-i][n-1-j] for i <= j, else 0
@@ -273,18 +450,30 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
 
   damp_kernel<<<1, 256, 0, st>>>(H, n, static_cast<double>(percdamp), stats);
   build_kernel<<<eb, 256, 0, st>>>(H, n, stats, A);
-  for (int k = 0; k < nb; ++k) {
-    potrf_kernel<<<1, 256, 0, st>>>(A, n, k, dinv, status_dev);
-    const int m = nb - k - 1;
-    if (m > 0) {
-      panel_kernel<<<m, 256, 0, st>>>(A, n, k, dinv);
-      trailing_kernel<<<m * (m + 1) / 2, 256, 0, st>>>(A, n, k);
+  for (int g0 = 0; g0 < nb; g0 += kGroup) {
+    const int g1 = g0 + kGroup < nb ? g0 + kGroup : nb;
+    for (int k = g0; k < g1; ++k) {
+      potrf_kernel<<<1, 256, 0, st>>>(A, n, k, dinv, status_dev);
+      const int below = nb - k - 1;
+      if (below > 0) panel_kernel<<<below, 256, 0, st>>>(A, n, k, dinv);
+      const int inner = g1 - k - 1;
+      if (below > 0 && inner > 0) group_update_kernel<<<dim3(below, inner), 256, 0, st>>>(A, n, k);
+    }
+    const int64_t e = static_cast<int64_t>(g1) * kNB;
+    if (e < n) {
+      const int nt = static_cast<int>((n - e + kT - 1) / kT);
+      rank_update_kernel<<<nt * (nt + 1) / 2, 256, 0, st>>>(A, n, e, static_cast<int64_t>(g0) * kNB, (g1 - g0) * kNB);
     }
   }
   seed_kernel<<<nb, 256, 0, st>>>(A, n, dinv);
-  for (int64_t s = kNB; s < n; s *= 2) {
+  if (n > kNB) {
+    const unsigned pairs = static_cast<unsigned>((n + 2 * kNB - 1) / (2 * kNB));
+    merge1_64_kernel<<<pairs, 256, 0, st>>>(A, n, T);
+    merge2_64_kernel<<<pairs, 256, 0, st>>>(A, n, T);
+  }
+  for (int64_t s = 2 * kNB; s < n; s *= 2) {
     const unsigned pairs = static_cast<unsigned>((n + 2 * s - 1) / (2 * s));
-    const unsigned tiles = static_cast<unsigned>((s / kNB) * (s / kNB));
+    const unsigned tiles = static_cast<unsigned>((s / kT) * (s / kT));
     merge1_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
     merge2_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
   }

@@ -18,7 +18,7 @@ def _hessian_f32(X):
     return O.hessian(to_np(X)).astype(np.float32)
 
 
-@pytest.mark.parametrize("n", [64, 256, 704, 1024])
+@pytest.mark.parametrize("n", [64, 128, 256, 704, 1024, 1152, 2048])
 def test_factor_matches_oracle(n):
     kind = "skew" if n == 704 else "normal"
     X = I.make_calib(I.CalibSpec(3 * n, n, "bf16", kind, max(1, n // 128), 30.0, 60.0, seed=31), "cuda")
