@@ -56,31 +56,35 @@ struct GroupParams {
   float rcp;    // correctly rounded 1/s, or 0 for a degenerate group (forces code 0)
 };
 
-__device__ __forceinline__ GroupParams group_params(float lo, float hi, float maxq) {
+// The correctly rounded binary32 quotient w / s without a division instruction sequence:
+// q0 = w * rcp is within an ulp of w / s, the residual w - s*q0 is exact in one FMA, and the
+// corrected q0 + residual*rcp is the correctly rounded quotient because rcp is the correctly
+// rounded reciprocal of s and the significand of s is not all ones (s is an fp16 value, or
+// one of the constants 7, 15): Markstein's division step.  With rcp == 0 (degenerate group)
+// the quotient is 0.
+__device__ __forceinline__ float quotient(float w, float s, float rcp) {
+  float q0 = __fmul_rn(w, rcp);
+  float r = __fmaf_rn(-s, q0, w);
+  return __fmaf_rn(r, rcp, q0);
+}
+
+// maxq is 2^bits - 1 and rcp_maxq the correctly rounded 1 / maxq (a compile-time constant at
+// the call sites): both divisions of the formula go through quotient() above, which returns
+// the correctly rounded binary32 quotient, so the result is that of true division.
+__device__ __forceinline__ GroupParams group_params(float lo, float hi, float maxq, float rcp_maxq) {
   lo = fminf(lo, 0.0f);
   hi = fmaxf(hi, 0.0f);
-  float s32 = __fdiv_rn(__fsub_rn(hi, lo), maxq);
+  float s32 = quotient(__fsub_rn(hi, lo), maxq, rcp_maxq);
   float s = __half2float(__float2half_rn(s32));
   GroupParams g;
   if (s == 0.0f || !isfinite(s)) {
     g.s = 1.0f; g.z = 0.0f; g.rcp = 0.0f;
   } else {
     g.s = s;
-    g.z = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), maxq) + 0.0f;   // + 0: never store -0
     g.rcp = __frcp_rn(s);
+    g.z = fminf(fmaxf(rintf(quotient(-lo, s, g.rcp)), 0.0f), maxq) + 0.0f;   // + 0: never store -0
   }
   return g;
-}
-
-// rint(w / s) with the binary32 quotient correctly rounded, without a division per weight:
-// q0 = w * rcp is within an ulp of w / s, the residual w - s*q0 is exact in one FMA, and the
-// corrected q0 + residual*rcp is the correctly rounded quotient because rcp is the correctly
-// rounded reciprocal of s and s, an fp16 value, never has an all-ones significand
-// (Markstein's division step).  With rcp == 0 (degenerate group) the quotient is 0.
-__device__ __forceinline__ float quotient(float w, float s, float rcp) {
-  float q0 = __fmul_rn(w, rcp);
-  float r = __fmaf_rn(-s, q0, w);
-  return __fmaf_rn(r, rcp, q0);
 }
 
 // Adding 1.5 * 2^23 rounds a float of magnitude < 2^22 to an integer (ties to even) held in

@@ -5,14 +5,27 @@
 //                     error e = (w - q) / U[i,i], and the update of the block's remaining
 //                     columns, w[j] -= e U[i,j].  The slab lives in shared memory; the 32
 //                     columns being worked on live in registers.
-//   trailing kernel - W[:, after the block] -= Err[out,128] * U[block rows, after the block],
-//                     an fp32 FFMA matrix product (the update feeds rounding decisions, so it
-//                     keeps full fp32 products).
+//   trailing update - W[:, after the block] -= Err[out,128] * U[block rows, after the block]
+//                     on the tensor cores with exactly sliced bf16 operands (gptq_tc.cu).
 // Rows are independent under per-OC grouping; under per-IC grouping a group couples g
 // consecutive rows of one column, which is why a CTA owns a whole 128-row slab.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace adadim {
+
+struct TrailPlan {
+  CUtensorMap e[3], u[3];
+  float* Wc;
+  int64_t rows_total, in;
+  int sm_count;
+};
+int trail_split_u(const float* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st);
+int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
+               const __nv_bfloat16* const u[3]);
+int trail_launch(const TrailPlan& plan, int i1, int* status_dev, cudaStream_t st);
 
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
@@ -46,7 +59,7 @@ init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const
 struct BlockArgs {
   float* Wc;                 // [ndim][out][in] working weights
   const float* U;            // [in][in]
-  float* Err;                // [ndim][out][128]
+  __nv_bfloat16* Ep[3];      // [ndim*out][128] errors as three fixed-point bf16 pieces
   double* loss_part;         // [ndim][out/128]
   adadim_qtensor q[2];       // outputs for the dimension(s) in flight
   int dim_of[2];             // grouping dimension of working copy d
@@ -58,6 +71,7 @@ template <int BITS, int G>
 __global__ void __launch_bounds__(kBlk, 1)
 block_kernel(const BlockArgs a) {
   constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr float rcp_maxq = 1.0f / maxq;            // correctly rounded at compile time
   constexpr int NG = kBlk / G;                       // per-IC groups in the slab
   extern __shared__ float sm[];
   float* Ws = sm;                                    // [128][129] slab of the working weights
@@ -113,7 +127,7 @@ block_kernel(const BlockArgs a) {
           } else {
             for (int k = 1; k < G; ++k) { float v = wrow[i + k]; mn = fminf(mn, v); mx = fmaxf(mx, v); }
           }
-          gp = group_params(mn, mx, maxq);
+          gp = group_params(mn, mx, maxq, rcp_maxq);
           int64_t idx = row * (a.in / G) + (a.i1 + i) / G;
           q.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
           q.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
@@ -135,7 +149,7 @@ block_kernel(const BlockArgs a) {
 #pragma unroll
           for (int k = 1; k < WPG; ++k) { mn = fminf(mn, slot[(w0 + k) * 2]); mx = fmaxf(mx, slot[(w0 + k) * 2 + 1]); }
         }
-        gp = group_params(mn, mx, maxq);
+        gp = group_params(mn, mx, maxq, rcp_maxq);
         if ((tid % G) == 0) {
           Ss[(tid / G) * kBlk + i] = __half_as_ushort(__float2half_rn(gp.s));
           Zs[(tid / G) * kBlk + i] = __half_as_ushort(__float2half_rn(gp.z));
@@ -185,8 +199,29 @@ block_kernel(const BlockArgs a) {
 
   // ---- outputs: errors (coalesced), per-IC parameters, loss ------------------------------
   __syncthreads();
-  float* Ed = a.Err + (static_cast<int64_t>(d) * a.out + row0) * kBlk;
-  for (int e = tid; e < kBlk * kBlk; e += kBlk) Ed[e] = Es[(e >> 7) * kPad + (e & 127)];
+  // errors as three fixed-point bf16 pieces on one grid per row (see gptq_tc.cu)
+  {
+    float m = 0.0f;
+    for (int k = 0; k < kBlk; ++k) m = fmaxf(m, fabsf(erow[k]));
+    int ex = (__float_as_int(m) >> 23) & 0xFF;
+    ex = ex < 32 ? 32 : (ex > 250 ? 250 : ex);
+    invd[tid] = __int_as_float((ex - 7) << 23);     // grid of this row (invd is free now)
+  }
+  __syncthreads();
+  const int64_t ebase = (static_cast<int64_t>(d) * a.out + row0) * kBlk;
+  for (int e = tid; e < kBlk * kBlk; e += kBlk) {
+    const int r = e >> 7;
+    const float v = Es[r * kPad + (e & 127)];
+    const float g = invd[r], inv = 1.0f / g;        // powers of two: exact
+    const float a0 = rintf(v * inv);
+    const float r1 = fmaf(-a0, g, v);
+    const float a1 = rintf(r1 * inv * 256.0f);
+    const float r2 = fmaf(-a1, g * (1.0f / 256.0f), r1);
+    const float a2 = rintf(r2 * inv * 65536.0f);
+    a.Ep[0][ebase + e] = __float2bfloat16_rn(a0 * g);
+    a.Ep[1][ebase + e] = __float2bfloat16_rn(a1 * g * (1.0f / 256.0f));
+    a.Ep[2][ebase + e] = __float2bfloat16_rn(a2 * g * (1.0f / 65536.0f));
+  }
   if (is_ic) {
     for (int e = tid; e < NG * kBlk; e += kBlk) {
       int64_t idx = (row0 / G + e / kBlk) * a.in + a.i1 + (e % kBlk);
@@ -199,56 +234,6 @@ block_kernel(const BlockArgs a) {
   if (lane == 0) lred[warp] = loss;
   __syncthreads();
   if (tid == 0) a.loss_part[static_cast<int64_t>(d) * (a.out / kBlk) + blockIdx.x] += (lred[0] + lred[1]) + (lred[2] + lred[3]);
-}
-
-// Wc[d][:, c0 + ...] -= Err[d] * U[i1 .. i1+127, c0 + ...], 128 x 128 output tile per CTA.
-__global__ void __launch_bounds__(256)
-trailing_kernel(float* __restrict__ Wc, const float* __restrict__ U, const float* __restrict__ Err, int64_t out,
-                int64_t in, int i1) {
-  __shared__ float sa[8][kBlk + 4];     // Err^T slice: [k][row]
-  __shared__ float sb[8][kBlk + 4];     // U slice:     [k][col]
-  const int64_t c0 = static_cast<int64_t>(i1) + kBlk + static_cast<int64_t>(blockIdx.x) * kBlk;
-  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kBlk;
-  float* Wd = Wc + static_cast<int64_t>(blockIdx.z) * out * in;
-  const float* Ed = Err + (static_cast<int64_t>(blockIdx.z) * out + r0) * kBlk;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  float acc[8][8] = {};
-  for (int k0 = 0; k0 < kBlk; k0 += 8) {
-    {
-      // Err tile: 128 rows x 8 k -> transposed; 256 threads x 4 elements
-      const int r = threadIdx.x >> 1, kq = (threadIdx.x & 1) * 4;
-      float4 v = *reinterpret_cast<const float4*>(Ed + r * kBlk + k0 + kq);
-      sa[kq + 0][r] = v.x; sa[kq + 1][r] = v.y; sa[kq + 2][r] = v.z; sa[kq + 3][r] = v.w;
-      const int kk = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4;
-      *reinterpret_cast<float4*>(&sb[kk][c4]) =
-          *reinterpret_cast<const float4*>(U + static_cast<int64_t>(i1 + k0 + kk) * in + c0 + c4);
-    }
-    __syncthreads();
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      float av[8], bv[8];
-      *reinterpret_cast<float4*>(av) = *reinterpret_cast<const float4*>(&sa[kk][ty * 4]);
-      *reinterpret_cast<float4*>(av + 4) = *reinterpret_cast<const float4*>(&sa[kk][64 + ty * 4]);
-      *reinterpret_cast<float4*>(bv) = *reinterpret_cast<const float4*>(&sb[kk][tx * 4]);
-      *reinterpret_cast<float4*>(bv + 4) = *reinterpret_cast<const float4*>(&sb[kk][64 + tx * 4]);
-#pragma unroll
-      for (int m = 0; m < 8; ++m)
-#pragma unroll
-        for (int n = 0; n < 8; ++n) acc[m][n] = fmaf(av[m], bv[n], acc[m][n]);
-    }
-    __syncthreads();
-  }
-#pragma unroll
-  for (int m = 0; m < 8; ++m) {
-    const int64_t r = r0 + (m < 4 ? ty * 4 + m : 64 + ty * 4 + (m - 4));
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      float4* p = reinterpret_cast<float4*>(Wd + r * in + c0 + h * 64 + tx * 4);
-      float4 v = *p;
-      v.x -= acc[m][h * 4 + 0]; v.y -= acc[m][h * 4 + 1]; v.z -= acc[m][h * 4 + 2]; v.w -= acc[m][h * 4 + 3];
-      *p = v;
-    }
-  }
 }
 
 __global__ void loss_kernel(const double* __restrict__ part, int ndim, int slabs, BlockArgs a, double* loss_out) {
@@ -274,12 +259,15 @@ int block_launch(const BlockArgs& a, int slabs, int ndim, cudaStream_t st) {
   return ADADIM_OK;
 }
 
-struct GptqLayout { size_t wc_off, err_off, loss_off, u_off, factor_off, total; };
+struct GptqLayout { size_t wc_off, err_off, err_piece, loss_off, up_off, up_piece, u_off, factor_off, total; };
 GptqLayout gptq_layout(int64_t out, int64_t in) {
   GptqLayout L;
   size_t off = 0;
   L.wc_off = off;     off += round_up(static_cast<size_t>(2) * out * in * 4, 256);
-  L.err_off = off;    off += round_up(static_cast<size_t>(2) * out * kBlk * 4, 256);
+  L.err_piece = round_up(static_cast<size_t>(2) * out * kBlk * 2, 1024);
+  L.err_off = off;    off += 3 * L.err_piece;
+  L.up_piece = round_up(static_cast<size_t>(in) * in * 2, 1024);
+  L.up_off = off;     off += 3 * L.up_piece;
   L.loss_off = off;   off += round_up(static_cast<size_t>(2) * (out / kBlk + 1) * 8, 256);
   L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 4, 256);
   L.factor_off = off; off += factor_workspace_bytes(in);
@@ -298,7 +286,13 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   BlockArgs a = {};
   a.Wc = reinterpret_cast<float*>(ws + L.wc_off);
-  a.Err = reinterpret_cast<float*>(ws + L.err_off);
+  const __nv_bfloat16* ep[3];
+  const __nv_bfloat16* up[3];
+  for (int k = 0; k < 3; ++k) {
+    a.Ep[k] = reinterpret_cast<__nv_bfloat16*>(ws + L.err_off + k * L.err_piece);
+    ep[k] = a.Ep[k];
+    up[k] = reinterpret_cast<__nv_bfloat16*>(ws + L.up_off + k * L.up_piece);
+  }
   a.loss_part = reinterpret_cast<double*>(ws + L.loss_off);
   a.out = out;
   a.in = in;
@@ -314,6 +308,9 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
     U = Uw;
   }
   a.U = U;
+  int rc0 = trail_split_u(U, in, const_cast<__nv_bfloat16*>(up[0]), const_cast<__nv_bfloat16*>(up[1]),
+                          const_cast<__nv_bfloat16*>(up[2]), st);
+  if (rc0 != ADADIM_OK) return rc0;
 
   const unsigned ib = static_cast<unsigned>((out * in / 8 + 255) / 256);
   if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, ndim, a.Wc);
@@ -321,6 +318,9 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   ADADIM_CUDA_TRY(cudaMemsetAsync(a.loss_part, 0, static_cast<size_t>(2) * (out / kBlk + 1) * 8, st));
 
   const int slabs = static_cast<int>(out / kBlk);
+  TrailPlan plan;
+  rc0 = trail_plan(&plan, a.Wc, static_cast<int64_t>(ndim) * out, in, ep, up);
+  if (rc0 != ADADIM_OK) return rc0;
   for (int i1 = 0; i1 < in; i1 += kBlk) {
     a.i1 = i1;
     int rc;
@@ -332,9 +332,10 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
                                                                                  : block_launch<4, 32>(a, slabs, ndim, st);
     }
     if (rc != ADADIM_OK) return rc;
-    const int64_t rest = in - i1 - kBlk;
-    if (rest > 0)
-      trailing_kernel<<<dim3(static_cast<unsigned>(rest / kBlk), slabs, ndim), 256, 0, st>>>(a.Wc, U, a.Err, out, in, i1);
+    if (in - i1 - kBlk > 0) {
+      rc = trail_launch(plan, i1, status_dev, st);
+      if (rc != ADADIM_OK) return rc;
+    }
   }
   if (gptq_loss != nullptr) loss_kernel<<<1, 32, 0, st>>>(a.loss_part, ndim, slabs, a, gptq_loss);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;

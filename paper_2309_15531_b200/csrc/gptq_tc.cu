@@ -1,0 +1,313 @@
+// GPTQ lazy-batch trailing update on the tensor cores (paper Section 2.2: the rounding error of
+// a block of columns is propagated to the columns not yet quantized):
+//     W[:, c0:] -= Err[rows,128] * U[i1:i1+128, c0:]
+// The update feeds later rounding decisions, so it needs fp32-grade accuracy, and the tensor
+// core's fp32 accumulation truncates (a bias of about half an ulp per addition, measured), which
+// summed over thousands of columns moved per-IC scales far more than an FFMA chain does.  The
+// operands are therefore sliced into three 8-bit fixed-point pieces on a common grid per Err row
+// and per U column of the block (x = p0 + p1 + p2, piece k a multiple of grid * 2^-8k).  Every
+// bf16 product of two leading pieces is then an integer multiple of one unit with at most 16
+// bits, a sum of 128 of them has at most 23 bits, and the accumulation is exact: nothing is
+// left to truncate.  The leading products go to one TMEM accumulator, the five smaller
+// product classes (2^-8 and 2^-16 of the result) to a second one, and the two are added in
+// fp32 in the epilogue.
+//
+// One CTA owns a 128-row block of the stacked working weights and a range of 128-column
+// tiles.  Its Err pieces (K = 128) stay in shared memory; U pieces stream through a ring of
+// 32-row slabs; two pairs of TMEM accumulators alternate so the read-modify-write of W of one
+// tile overlaps the MMAs of the next.
+#include <cuda_bf16.h>
+
+#include "umma.cuh"
+
+namespace adadim {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr uint32_t kAPiece = 128 * 64 * 2;          // one Err piece, one 64-deep half of K: 16 KB
+constexpr uint32_t kABytes = 6 * kAPiece;           // 3 pieces x 2 halves
+constexpr int kTileN = 128;
+constexpr uint32_t kBPiece = kTileN * 32 * 2;       // one U piece, 32 k-rows x 128 columns: 8 KB
+constexpr uint32_t kBStage = 3 * kBPiece;           // 24 KB
+constexpr int kBStages = 4;
+constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 1024 + 256;
+
+struct TrailParams {
+  float* Wc;            // [rows_total][in] stacked working weights
+  int64_t in;
+  int64_t c0;           // first column to update
+  int i1;               // first row of U's block
+  int ntiles;           // 128-column tiles from c0
+  int* status_dev;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ CUtensorMap tmE1,
+             const __grid_constant__ CUtensorMap tmE2, const __grid_constant__ CUtensorMap tmU0,
+             const __grid_constant__ CUtensorMap tmU1, const __grid_constant__ CUtensorMap tmU2,
+             const TrailParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a_smem = smem;
+  uint8_t* b_smem = smem + kABytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + kBStages * kBStage);
+  uint64_t* a_full = bars;
+  uint64_t* b_full = bars + 1;                      // [kBStages]
+  uint64_t* b_empty = b_full + kBStages;            // [kBStages]
+  uint64_t* acc_full = b_empty + kBStages;          // [2]
+  uint64_t* acc_empty = acc_full + 2;               // [2]
+  uint64_t* drain = acc_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // this CTA's tiles: an even share of [0, ntiles)
+  const int per = (p.ntiles + gridDim.x - 1) / gridDim.x;
+  const int t0 = blockIdx.x * per;
+  const int t1 = min(t0 + per, p.ntiles);
+  const int mrow = blockIdx.y * 128;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(a_full, 1);
+    for (int s = 0; s < kBStages; ++s) { ptx::mbar_init(&b_full[s], 1); ptx::mbar_init(&b_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { ptx::mbar_init(&acc_full[s], 1); ptx::mbar_init(&acc_empty[s], 4); }
+    ptx::mbar_init(drain, 1);
+    *dead = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0 && t0 < t1) {
+      const CUtensorMap* tmE[3] = {&tmE0, &tmE1, &tmE2};
+      const CUtensorMap* tmU[3] = {&tmU0, &tmU1, &tmU2};
+      ptx::mbar_arrive_expect_tx(a_full, kABytes);
+      for (int pc = 0; pc < 3; ++pc)
+        for (int kh = 0; kh < 2; ++kh)
+          ptx::tma_load_2d(a_smem + (pc * 2 + kh) * kAPiece, tmE[pc], kh * 64, mrow, a_full);
+      int stage = 0;
+      uint32_t phase = 0;
+      int last_phase[kBStages];
+      for (int s = 0; s < kBStages; ++s) last_phase[s] = -1;
+      for (int t = t0; t < t1 && !*dead; ++t) {
+        const int col = static_cast<int>(p.c0) + t * kTileN;
+        for (int kc = 0; kc < 4; ++kc) {
+          if (!ptx::mbar_wait(&b_empty[stage], phase ^ 1u, dead, p.status_dev)) break;
+          ptx::mbar_arrive_expect_tx(&b_full[stage], kBStage);
+          last_phase[stage] = static_cast<int>(phase);
+          uint8_t* dst = b_smem + stage * kBStage;
+          for (int pc = 0; pc < 3; ++pc)
+            for (int j = 0; j < kTileN / 64; ++j)
+              ptx::tma_load_2d(dst + pc * kBPiece + j * (32 * 128), tmU[pc], col + j * 64, p.i1 + kc * 32, &b_full[stage]);
+          if (++stage == kBStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (*dead) {
+        // a wait ran out somewhere: let the copies already issued land before shared memory goes away
+        const long long c0 = clock64();
+        while (!ptx::mbar_try_wait(a_full, 0) && clock64() - c0 < ptx::kWaitLimit) {}
+        for (int s = 0; s < kBStages; ++s) {
+          if (last_phase[s] < 0) continue;
+          const long long c1 = clock64();
+          while (!ptx::mbar_try_wait(&b_full[s], static_cast<uint32_t>(last_phase[s])) && clock64() - c1 < ptx::kWaitLimit) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && t0 < t1) {
+      constexpr uint32_t idesc = ptx::idesc_bf16(128, kTileN, false, true);
+      constexpr uint64_t adesc = ptx::smem_desc_sw128(16, 1024);          // K-major, 8-row groups 1024 B apart
+      constexpr uint64_t bdesc = ptx::smem_desc_sw128(32 * 128, 1024);    // MN-major, 64-column blocks 4 KB apart
+      bool ok = ptx::mbar_wait(a_full, 0, dead, p.status_dev);
+      int stage = 0;
+      uint32_t phase = 0, acc_phase[2] = {0, 0};
+      for (int t = t0; t < t1 && ok; ++t) {
+        const int buf = (t - t0) & 1;
+        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase[buf] ^ 1u, dead, p.status_dev)) break;
+        ptx::tc_fence_after_sync();
+        for (int kc = 0; kc < 4; ++kc) {
+          if (!ptx::mbar_wait(&b_full[stage], phase, dead, p.status_dev)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t a_addr = ptx::smem_addr(a_smem) + (kc >> 1) * kAPiece + (kc & 1) * 64;
+          const uint32_t b_addr = ptx::smem_addr(b_smem + stage * kBStage);
+#pragma unroll
+          for (int k16 = 0; k16 < 2; ++k16) {
+#pragma unroll
+            for (int pr = 0; pr < 6; ++pr) {
+              // (Err piece, U piece) with piece indices summing to at most 2
+              const int pa = pr == 0 ? 0 : pr == 1 ? 0 : pr == 2 ? 1 : pr == 3 ? 0 : pr == 4 ? 1 : 2;
+              const int pb = pr == 0 ? 0 : pr == 1 ? 1 : pr == 2 ? 0 : pr == 3 ? 2 : pr == 4 ? 1 : 0;
+              // leading product -> exact accumulator; the rest -> the second one
+              const uint32_t acc = tmem_base + buf * 256 + (pr == 0 ? 0 : kTileN);
+              const bool first = (kc | k16) == 0 && pr <= 1;
+              ptx::mma_f16(acc, ptx::with_start(adesc, a_addr + pa * 2 * kAPiece + k16 * 32),
+                           ptx::with_start(bdesc, b_addr + pb * kBPiece + k16 * (16 * 128)), idesc, !first);
+            }
+          }
+          ptx::mma_commit(&b_empty[stage]);
+          if (++stage == kBStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::mma_commit(&acc_full[buf]);
+        acc_phase[buf] ^= 1u;
+      }
+      if (*dead) {
+        ptx::mma_commit(drain);
+        const long long c0 = clock64();
+        while (!ptx::mbar_try_wait(drain, 0) && clock64() - c0 < ptx::kWaitLimit) {}
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    uint32_t acc_phase[2] = {0, 0};
+    float* wrow = p.Wc + (static_cast<int64_t>(mrow) + q * 32 + lane) * p.in;
+    for (int t = t0; t < t1; ++t) {
+      const int buf = (t - t0) & 1;
+      if (!ptx::mbar_wait(&acc_full[buf], acc_phase[buf], dead, p.status_dev)) break;
+      ptx::tc_fence_after_sync();
+      const int64_t col = p.c0 + static_cast<int64_t>(t) * kTileN;
+#pragma unroll 1
+      for (int c = 0; c < kTileN / 32; ++c) {
+        float v[32], v2[32];
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + c * 32;
+        ptx::tmem_ld32(taddr, v);
+        ptx::tmem_ld32(taddr + kTileN, v2);
+        const int64_t j0 = col + c * 32;
+        if (j0 < p.in) {                      // in % 128 == 0: a 32-column chunk is all in or all out
+          float4* w4 = reinterpret_cast<float4*>(wrow + j0);
+          float4 w[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) w[k] = w4[k];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            w[k].x -= v[4 * k] + v2[4 * k];         w[k].y -= v[4 * k + 1] + v2[4 * k + 1];
+            w[k].z -= v[4 * k + 2] + v2[4 * k + 2]; w[k].w -= v[4 * k + 3] + v2[4 * k + 3];
+            w4[k] = w[k];
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+      acc_phase[buf] ^= 1u;
+    }
+  }
+
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Fixed-point slicing shared by both operands: with ex the biased exponent of the largest
+// magnitude of a slice group (clamped so that all three grids are normal numbers),
+// grid = 2^(ex - 134), and x = a0*grid + a1*grid/256 + a2*grid/65536 with integers |a0| <= 256,
+// |a1|, |a2| <= 128 (each product a*grid is exact in bf16).
+struct SliceGrid { float g, inv; };
+__device__ __forceinline__ SliceGrid slice_grid(float maxabs) {
+  int ex = (__float_as_int(maxabs) >> 23) & 0xFF;
+  ex = ex < 32 ? 32 : (ex > 250 ? 250 : ex);
+  SliceGrid s;
+  s.g = __int_as_float((ex - 7) << 23);             // 2^(ex - 127 - 7)
+  s.inv = __int_as_float((254 - (ex - 7)) << 23);   // 1 / g
+  return s;
+}
+__device__ __forceinline__ void slice3(float x, SliceGrid s, __nv_bfloat16& p0, __nv_bfloat16& p1, __nv_bfloat16& p2) {
+  const float a0 = rintf(x * s.inv);
+  const float r1 = fmaf(-a0, s.g, x);                       // exact
+  const float a1 = rintf(r1 * s.inv * 256.0f);
+  const float r2 = fmaf(-a1, s.g * (1.0f / 256.0f), r1);    // exact
+  const float a2 = rintf(r2 * s.inv * 65536.0f);
+  p0 = __float2bfloat16_rn(a0 * s.g);
+  p1 = __float2bfloat16_rn(a1 * s.g * (1.0f / 256.0f));
+  p2 = __float2bfloat16_rn(a2 * s.g * (1.0f / 65536.0f));
+}
+
+// U pieces: one grid per (128-row block b, column c).  Only columns right of the block are
+// ever read by the trailing update, so only those are written.
+__global__ void __launch_bounds__(128)
+slice_u_kernel(const float* __restrict__ U, int64_t in, __nv_bfloat16* __restrict__ p0, __nv_bfloat16* __restrict__ p1,
+               __nv_bfloat16* __restrict__ p2) {
+  const int b = blockIdx.y;
+  if (static_cast<int>(blockIdx.x) <= b) return;
+  const int64_t c = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
+  const float* src = U + static_cast<int64_t>(b) * 128 * in + c;
+  float v[128];
+  float m = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 128; ++i) { v[i] = src[static_cast<int64_t>(i) * in]; m = fmaxf(m, fabsf(v[i])); }
+  const SliceGrid sg = slice_grid(m);
+#pragma unroll
+  for (int i = 0; i < 128; ++i) {
+    __nv_bfloat16 a, bb, cc;
+    slice3(v[i], sg, a, bb, cc);
+    const int64_t idx = (static_cast<int64_t>(b) * 128 + i) * in + c;
+    p0[idx] = a; p1[idx] = bb; p2[idx] = cc;
+  }
+}
+
+}  // namespace
+
+// Host-side state of one GPTQ call's trailing updates: the six tensor maps never change
+// between blocks, only the coordinates do.
+struct TrailPlan {
+  CUtensorMap e[3], u[3];
+  float* Wc;
+  int64_t rows_total, in;
+  int sm_count;
+};
+
+int trail_split_u(const float* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st) {
+  const unsigned nb = static_cast<unsigned>(in / 128);
+  if (nb > 1) slice_u_kernel<<<dim3(nb, nb - 1), 128, 0, st>>>(U, in, u0, u1, u2);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
+               const __nv_bfloat16* const u[3]) {
+  plan->Wc = Wc;
+  plan->rows_total = rows_total;
+  plan->in = in;
+  for (int k = 0; k < 3; ++k) {
+    int rc = make_tmap_bf16(&plan->e[k], e[k], 128, static_cast<uint64_t>(rows_total), 256, 128);
+    if (rc != ADADIM_OK) return rc;
+    rc = make_tmap_bf16(&plan->u[k], u[k], static_cast<uint64_t>(in), static_cast<uint64_t>(in),
+                        static_cast<uint64_t>(in) * 2, 32);
+    if (rc != ADADIM_OK) return rc;
+  }
+  int dev = 0;
+  ADADIM_CUDA_TRY(cudaGetDevice(&dev));
+  ADADIM_CUDA_TRY(cudaDeviceGetAttribute(&plan->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  ADADIM_CUDA_TRY(cudaFuncSetAttribute(trail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(kSmemBytes)));
+  return ADADIM_OK;
+}
+
+int trail_launch(const TrailPlan& plan, int i1, int* status_dev, cudaStream_t st) {
+  TrailParams p;
+  p.Wc = plan.Wc;
+  p.in = plan.in;
+  p.c0 = static_cast<int64_t>(i1) + 128;
+  p.i1 = i1;
+  p.ntiles = static_cast<int>((plan.in - p.c0 + kTileN - 1) / kTileN);
+  p.status_dev = status_dev;
+  if (p.ntiles <= 0) return ADADIM_OK;
+  const int mblocks = static_cast<int>(plan.rows_total / 128);
+  int nsplit = plan.sm_count / mblocks;
+  if (nsplit < 1) nsplit = 1;
+  if (nsplit > p.ntiles) nsplit = p.ntiles;
+  trail_kernel<<<dim3(nsplit, mblocks), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],
+                                                                      plan.u[1], plan.u[2], p);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
+}  // namespace adadim

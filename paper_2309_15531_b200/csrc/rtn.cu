@@ -32,6 +32,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
                 adadim_qtensor qoc, adadim_qtensor qic) {
   constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr float rcp_maxq = 1.0f / maxq;            // correctly rounded at compile time
   constexpr int NG = kTile / G;               // per-IC groups stacked in one tile
   constexpr int PPG = kPasses / NG;           // passes per such group
   constexpr int LANES_PER_OCG = G / 8;        // threads sharing one per-OC group
@@ -99,7 +100,7 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
         mn = fminf(mn, s_mn[gi][wv][c]);
         mx = fmaxf(mx, s_mx[gi][wv][c]);
       }
-      GroupParams gp = group_params(mn, mx, maxq);
+      GroupParams gp = group_params(mn, mx, maxq, rcp_maxq);
       s_s[gi][c] = gp.rcp == 0.0f ? 0.0f : gp.s;      // 0 marks a degenerate group
       s_z[gi][c] = gp.z;
       int64_t grow = r0 / G + gi;
@@ -140,7 +141,7 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
           mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, m));
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
         }
-        GroupParams gp = group_params(mn, mx, maxq);
+        GroupParams gp = group_params(mn, mx, maxq, rcp_maxq);
         if (ok && (colvec % LANES_PER_OCG) == 0) {
           int64_t idx = row * (in / G) + col / G;
           qoc.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));

@@ -87,7 +87,7 @@ def _gptq_case(W, X, bits, group, rows=None):
 
 @pytest.mark.parametrize("bits,group", [(3, 128), (4, 128), (3, 64), (4, 32)])
 def test_small_layers(bits, group):
-    W = I.make_weight(I.WeightSpec(256, 512, "f16", 0.02, 0.001, seed=41), "cuda")
+    W = I.make_weight(I.WeightSpec(512, 512, "f16", 0.02, 0.001, seed=41), "cuda")
     X = I.make_calib(I.CalibSpec(4096, 512, "bf16", "normal", 3, 50.0, 100.0, seed=42), "cuda")
     _gptq_case(W, X, bits, group)
 
