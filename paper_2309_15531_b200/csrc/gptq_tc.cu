@@ -170,27 +170,26 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
     float* wrow = p.Wc + (static_cast<int64_t>(mrow) + q * 32 + lane) * p.in;
     for (int t = t0; t < t1; ++t) {
       const int buf = (t - t0) & 1;
+      // The tile's slice of W does not depend on the MMAs: fetch it while they run.
+      // (in % 128 == 0 and c0 % 128 == 0, so every tile lies wholly inside the matrix.)
+      float4* w4 = reinterpret_cast<float4*>(wrow + p.c0 + static_cast<int64_t>(t) * kTileN);
+      float4 w[kTileN / 4];
+#pragma unroll
+      for (int k = 0; k < kTileN / 4; ++k) w[k] = w4[k];
       if (!ptx::mbar_wait(&acc_full[buf], acc_phase[buf], dead, p.status_dev)) break;
       ptx::tc_fence_after_sync();
-      const int64_t col = p.c0 + static_cast<int64_t>(t) * kTileN;
-#pragma unroll 1
+#pragma unroll
       for (int c = 0; c < kTileN / 32; ++c) {
         float v[32], v2[32];
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + c * 32;
         ptx::tmem_ld32(taddr, v);
         ptx::tmem_ld32(taddr + kTileN, v2);
-        const int64_t j0 = col + c * 32;
-        if (j0 < p.in) {                      // in % 128 == 0: a 32-column chunk is all in or all out
-          float4* w4 = reinterpret_cast<float4*>(wrow + j0);
-          float4 w[8];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) w[k] = w4[k];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            w[k].x -= v[4 * k] + v2[4 * k];         w[k].y -= v[4 * k + 1] + v2[4 * k + 1];
-            w[k].z -= v[4 * k + 2] + v2[4 * k + 2]; w[k].w -= v[4 * k + 3] + v2[4 * k + 3];
-            w4[k] = w[k];
-          }
+        for (int k = 0; k < 8; ++k) {
+          float4 x = w[c * 8 + k];
+          x.x -= v[4 * k] + v2[4 * k];         x.y -= v[4 * k + 1] + v2[4 * k + 1];
+          x.z -= v[4 * k + 2] + v2[4 * k + 2]; x.w -= v[4 * k + 3] + v2[4 * k + 3];
+          w4[c * 8 + k] = x;
         }
       }
       ptx::tc_fence_before_sync();
