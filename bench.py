@@ -106,7 +106,7 @@ def launches_per_step(out: int, inp: int) -> int:
     gptq = 1 + 1 + blocks + (blocks - 1) + 1           # init, U slicing, block kernels, trailing kernels, loss
     hessian = 2 if inp > 256 else 1
     rtn = 1
-    score = 2 + 1 + 1 + 1
+    score = 2 + 1 + 1                                  # two difference kernels, Gram product, finalize
     return hessian + rtn + score + factor + gptq + score
 
 
@@ -255,7 +255,7 @@ def run_ours(args):
     tile = 256
     hess_flops = ntok * inp * (inp + tile)              # lower-triangle tiles of the symmetric product
     rtn_bytes = weights * (2 + 2 * (BITS / 8 + 4 / GROUP))
-    score_flops = 2 * (2 * out) * inp * inp             # both dims stacked (algorithmic: one pass over H)
+    score_flops = 2 * out * inp * (inp + tile)           # D^T D on lower-triangle tiles, both dims
     factor_flops = 2 * inp ** 3 / 3                     # Cholesky + triangular inverse
     gptq_flops = 2 * (out * inp * inp)                  # trailing + in-block updates, both dims
     roof_all = {

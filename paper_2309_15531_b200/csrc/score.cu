@@ -1,19 +1,19 @@
 // Reconstruction-error scorer and selection (paper Section 3.3, Eq. 1; Appendix B):
 //   E_dim = || X (W - Q_dim)^T ||_F^2 = 1/2 trace(D_dim H D_dim^T),  D_dim = W - Q_dim,
 //   chosen = IC iff E_ic < E_oc.
-// Steps: (1) D for both dimensions, stacked [OC rows; IC rows], rounded to bf16;
-// (2) H split into bf16 high and low parts (H = Hhi + Hlo to about 2^-17 relative);
-// (3) tensor-core contraction S = D (Hhi + Hlo) with sum(D .* S) taken per tile (tc_gemm.cu);
-// (4) fixed-order reduction of the per-tile partials and the comparison.
+// Steps: (1) D for each dimension, rounded to bf16;
+// (2) tensor-core symmetric product D^T D on lower-triangle tiles with sum(H .* D^T D) taken per
+//     tile against the fp32 H (tc_gemm.cu): half the multiplications of D H, and H stays exact;
+// (3) fixed-order reduction of the per-tile partials and the comparison.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
 
 namespace adadim {
 
-int score_gemm_launch(const __nv_bfloat16* D, int64_t m_total, int64_t in, const __nv_bfloat16* Hhi,
-                      const __nv_bfloat16* Hlo, double* partial, int* status_dev, cudaStream_t st);
-int score_tiles(int64_t m_total, int64_t in);
+int gram_launch(const __nv_bfloat16* D0, const __nv_bfloat16* D1, int64_t rows, int64_t in, const float* H,
+                double* partial, int* status_dev, cudaStream_t st);
+int gram_tiles(int64_t in);
 
 namespace {
 
@@ -64,35 +64,18 @@ diff_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int g
   }
 }
 
+// partial is [tiles][2 halves][4]; tiles below `tiles_first` belong to the first scored
+// dimension.  Sums are taken in a fixed order.
 __global__ void __launch_bounds__(256)
-split_kernel(const float* __restrict__ H, int64_t n, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
-  int64_t i = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
-  if (i >= n) return;
-  float4 h = *reinterpret_cast<const float4*>(H + i);
-  float v[4] = {h.x, h.y, h.z, h.w};
-  __nv_bfloat16 a[4], b[4];
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    a[k] = __float2bfloat16_rn(v[k]);
-    b[k] = __float2bfloat16_rn(v[k] - __bfloat162float(a[k]));
-  }
-  *reinterpret_cast<uint2*>(hi + i) = *reinterpret_cast<uint2*>(a);
-  *reinterpret_cast<uint2*>(lo + i) = *reinterpret_cast<uint2*>(b);
-}
-
-// partial is [tiles][2 halves][4]; a half is a 128-row block; row blocks below `blocks_first`
-// belong to the first stacked dimension.  Sums are taken in a fixed order.
-__global__ void __launch_bounds__(256)
-finalize_kernel(const double* __restrict__ partial, int num_tiles, int tiles_n, int blocks_first,
+finalize_kernel(const double* __restrict__ partial, int num_tiles, int tiles_first,
                 int first_dim, bool have_second, double* err, int* chosen, int* status_dev) {
   __shared__ double red[2][256];
   double acc[2] = {0.0, 0.0};
   for (int e = threadIdx.x; e < num_tiles * 2; e += 256) {
-    int tile = e >> 1, half = e & 1;
-    int block_row = (tile / tiles_n) * 2 + half;
+    const int tile = e >> 1;
     const double* pp = partial + static_cast<int64_t>(e) * 4;
     double s = (pp[0] + pp[1]) + (pp[2] + pp[3]);
-    acc[block_row < blocks_first ? 0 : 1] += s;
+    acc[tile < tiles_first ? 0 : 1] += s;
   }
   red[0][threadIdx.x] = acc[0];
   red[1][threadIdx.x] = acc[1];
@@ -128,15 +111,13 @@ void diff_launch(const T* W, int64_t out, int64_t in, int64_t ldw, int bits, int
 }
 
 struct ScoreLayout {
-  size_t d_off, hi_off, lo_off, part_off, total;
+  size_t d_off, part_off, total;
 };
 ScoreLayout score_layout(int64_t out, int64_t in) {
   ScoreLayout L;
   size_t off = 0;
   L.d_off = off;    off += round_up(static_cast<size_t>(2 * out) * in * 2, 256);
-  L.hi_off = off;   off += round_up(static_cast<size_t>(in) * in * 2, 256);
-  L.lo_off = off;   off += round_up(static_cast<size_t>(in) * in * 2, 256);
-  L.part_off = off; off += round_up(static_cast<size_t>(score_tiles(2 * out, in)) * 8 * sizeof(double), 256);
+  L.part_off = off; off += round_up(static_cast<size_t>(2 * gram_tiles(in)) * 8 * sizeof(double), 256);
   L.total = off;
   return L;
 }
@@ -151,8 +132,6 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
   ScoreLayout L = score_layout(out, in);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   __nv_bfloat16* D = reinterpret_cast<__nv_bfloat16*>(ws + L.d_off);
-  __nv_bfloat16* Hhi = reinterpret_cast<__nv_bfloat16*>(ws + L.hi_off);
-  __nv_bfloat16* Hlo = reinterpret_cast<__nv_bfloat16*>(ws + L.lo_off);
   double* partial = reinterpret_cast<double*>(ws + L.part_off);
 
   const adadim_qtensor* qs[2] = {q_oc, q_ic};
@@ -166,14 +145,12 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
     else diff_launch(static_cast<const float*>(W), out, in, ldw, bits, group, d == 1, *qs[d], dst, st);
     rows += out;
   }
-  const int64_t n = in * in;
-  split_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, st>>>(H, n, Hhi, Hlo);
   if (cudaGetLastError() != cudaSuccess) return ADADIM_ERR_CUDA;
-  int rc = score_gemm_launch(D, rows, in, Hhi, Hlo, partial, status_dev, st);
+  int rc = gram_launch(D, have_second ? D + out * in : nullptr, out, in, H, partial, status_dev, st);
   if (rc != ADADIM_OK) return rc;
-  const int tiles_n = static_cast<int>((in + 255) / 256);
-  finalize_kernel<<<1, 256, 0, st>>>(partial, score_tiles(rows, in), tiles_n, static_cast<int>(out / 128), first_dim,
-                                     have_second, err, chosen, status_dev);
+  const int tiles = gram_tiles(in);
+  finalize_kernel<<<1, 256, 0, st>>>(partial, tiles * (have_second ? 2 : 1), tiles, first_dim, have_second, err, chosen,
+                                     status_dev);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 

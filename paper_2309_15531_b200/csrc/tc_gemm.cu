@@ -2,8 +2,9 @@
 //   * calibration Hessian  H += 2 X^T X  (paper Section 4.4; Section 2.2) as a symmetric
 //     rank-k update over the tokens, lower-triangle 256 x 256 output tiles only (a copy kernel
 //     mirrors them into the upper triangle afterwards);
-//   * the reconstruction-error contraction  S = D H  of  1/2 trace(D H D^T)  (Section 3.3, Eq. 1),
-//     with the sum over D .* S taken in the epilogue.
+//   * the reconstruction-error contraction of  1/2 trace(D H D^T) = 1/2 sum(H .* D^T D)
+//     (Section 3.3, Eq. 1): D^T D is the same kind of symmetric product, over the rows of D, and
+//     the sum against the fp32 H is taken in the epilogue, so H is never rounded.
 // One CTA owns a 256 x 256 output tile as two 128 x 256 fp32 accumulators filling all 512
 // TMEM columns.  Warp 0 feeds the ring with TMA, one thread of warp 1 issues the MMAs, warps
 // 2..5 drain the accumulators.  All CTAs sweep the reduction dimension from the start at the
@@ -53,7 +54,7 @@ int make_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner, uint64_t 
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-enum class Mode { kHessian, kScore };
+enum class Mode { kHessian, kGram };
 
 struct TcParams {
   int num_tiles;            // output tiles (256 x 256) to process
@@ -63,10 +64,8 @@ struct TcParams {
   // Hessian
   float* H;
   int64_t in;               // H is [in][in]; also the column count of D
-  // Score
-  const __nv_bfloat16* D;   // [m_total][in]
-  int64_t m_total;
-  int tiles_n;              // column tiles of S
+  // Gram (scorer): tiles [0, tiles_per_dim) belong to the first D, the rest to the second
+  int tiles_per_dim;
   double* partial;          // [num_tiles][2 halves][4 warps]
 };
 
@@ -76,7 +75,7 @@ constexpr uint32_t kOperandBytes = 256 * kKT * 2;   // one 256-wide bf16 operand
 
 template <Mode MODE> struct TcCfg;
 template <> struct TcCfg<Mode::kHessian> { static constexpr int NB = 1, STAGES = 3; static constexpr bool MN = true; };
-template <> struct TcCfg<Mode::kScore>   { static constexpr int NB = 2, STAGES = 2; static constexpr bool MN = false; };
+template <> struct TcCfg<Mode::kGram>    { static constexpr int NB = 1, STAGES = 3; static constexpr bool MN = true; };
 
 template <Mode MODE>
 constexpr size_t tc_smem_bytes() {
@@ -121,7 +120,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&tmA);
     ptx::tma_prefetch_desc(&tmB0);
-    if (NB == 2) ptx::tma_prefetch_desc(&tmB1);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, 512);
@@ -141,29 +139,24 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       for (int s = 0; s < STAGES; ++s) last_phase[s] = -1;
       for (int t = blockIdx.x; t < p.num_tiles && !*dead; t += gridDim.x) {
         int rb, cb;
-        if (MODE == Mode::kHessian) tri_coords(t, rb, cb); else { rb = t / p.tiles_n; cb = t % p.tiles_n; }
-        const bool shared_operand = (MODE == Mode::kHessian) && rb == cb;   // B is A on the diagonal
+        const int which = MODE == Mode::kGram ? t / p.tiles_per_dim : 0;     // which stacked matrix
+        tri_coords(MODE == Mode::kGram ? t % p.tiles_per_dim : t, rb, cb);
+        const CUtensorMap* tm = which == 0 ? &tmA : &tmB0;
+        const bool shared_operand = rb == cb;                              // B is A on the diagonal
         for (int k = 0; k < p.num_k; ++k) {
           if (!ptx::mbar_wait(&empty[stage], phase ^ 1u, dead, p.status_dev)) break;
           uint8_t* a_dst = smem + stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + kOperandBytes;
           ptx::mbar_arrive_expect_tx(&full[stage], shared_operand ? kOperandBytes : STAGE_BYTES);
           last_phase[stage] = static_cast<int>(phase);
-          if (MODE == Mode::kHessian) {
-            // X is [tokens][in]: boxes of 64 channels x 64 tokens, channels contiguous (MN-major)
+          // the matrix is [tokens][in]: boxes of 64 channels x 64 tokens, channels contiguous (MN-major)
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            ptx::tma_load_2d(a_dst + j * (kKT * 128), tm, rb * 256 + j * 64, k * kKT, &full[stage]);
+          if (!shared_operand) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              ptx::tma_load_2d(a_dst + j * (kKT * 128), &tmA, rb * 256 + j * 64, k * kKT, &full[stage]);
-            if (!shared_operand) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j)
-                ptx::tma_load_2d(b_dst + j * (kKT * 128), &tmB0, cb * 256 + j * 64, k * kKT, &full[stage]);
-            }
-          } else {
-            // D is [rows][in] and H is [in][in]: boxes of 64 reduction elements x 256 rows (K-major)
-            ptx::tma_load_2d(a_dst, &tmA, k * kKT, rb * 256, &full[stage]);
-            ptx::tma_load_2d(b_dst, &tmB0, k * kKT, cb * 256, &full[stage]);
-            ptx::tma_load_2d(b_dst + kOperandBytes, &tmB1, k * kKT, cb * 256, &full[stage]);
+              ptx::tma_load_2d(b_dst + j * (kKT * 128), tm, cb * 256 + j * 64, k * kKT, &full[stage]);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -190,8 +183,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       uint32_t phase = 0, acc_phase = 0;
       for (int t = blockIdx.x; t < p.num_tiles && !*dead; t += gridDim.x) {
         int rb, cb;
-        if (MODE == Mode::kHessian) tri_coords(t, rb, cb); else { rb = t / p.tiles_n; cb = t % p.tiles_n; }
-        const bool shared_operand = (MODE == Mode::kHessian) && rb == cb;
+        tri_coords(MODE == Mode::kGram ? t % p.tiles_per_dim : t, rb, cb);
+        const bool shared_operand = rb == cb;
         bool ok = true;
         for (int kc = 0; kc < p.num_k && ok; kc += p.k_chunk) {
           if (!ptx::mbar_wait(acc_empty, acc_phase ^ 1u, dead, p.status_dev)) { ok = false; break; }
@@ -236,7 +229,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     uint32_t acc_phase = 0;
     for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
       int rb, cb;
-      if (MODE == Mode::kHessian) tri_coords(t, rb, cb); else { rb = t / p.tiles_n; cb = t % p.tiles_n; }
+      tri_coords(MODE == Mode::kGram ? t % p.tiles_per_dim : t, rb, cb);
       bool live = true;
       for (int kc = 0; kc < p.num_k; kc += p.k_chunk) {
       live = ptx::mbar_wait(acc_full, acc_phase, dead, p.status_dev);
@@ -265,21 +258,20 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               }
             }
           } else {
-            if (i < p.m_total && j0 < p.in) {       // in % 64 == 0: a 32-column chunk is all in or out
-              const uint4* dp = reinterpret_cast<const uint4*>(p.D + i * p.in + j0);
+            // sum of H .* (D^T D) over this warp's rows of the tile; tiles below the diagonal
+            // stand for their mirror image too
+            if (i < p.in) {
+              const float* hrow = p.H + i * p.in + j0;
               float acc = 0.0f;
 #pragma unroll
-              for (int k8 = 0; k8 < 4; ++k8) {
-                uint4 raw = dp[k8];
-                const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                  float2 f = __bfloat1622float2(d2[m]);
-                  acc = fmaf(f.x, v[k8 * 8 + 2 * m], acc);
-                  acc = fmaf(f.y, v[k8 * 8 + 2 * m + 1], acc);
+              for (int k4 = 0; k4 < 8; ++k4) {
+                if (j0 + k4 * 4 < p.in) {
+                  const float4 h = *reinterpret_cast<const float4*>(hrow + k4 * 4);
+                  acc = fmaf(h.x, v[k4 * 4 + 0], acc); acc = fmaf(h.y, v[k4 * 4 + 1], acc);
+                  acc = fmaf(h.z, v[k4 * 4 + 2], acc); acc = fmaf(h.w, v[k4 * 4 + 3], acc);
                 }
               }
-              part[a] += static_cast<double>(acc);
+              part[a] += static_cast<double>(acc) * (rb == cb ? 1.0 : 2.0);
             }
           }
         }
@@ -287,7 +279,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty);
-      if (MODE == Mode::kScore) {
+      if (MODE == Mode::kGram) {
         // one partial per (tile, 128-row half, warp): no cross-warp synchronisation needed
 #pragma unroll
         for (int a = 0; a < 2; ++a) {
@@ -423,32 +415,33 @@ int hessian_f32_launch(const float* X, int64_t n_tokens, int64_t in, int64_t ldx
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 
-// S = D * (Hhi + Hlo); partial[tile][half][warp] = that warp's share of the sum of D .* S over the
-// tile's 128-row half.
-int score_gemm_launch(const __nv_bfloat16* D, int64_t m_total, int64_t in, const __nv_bfloat16* Hhi,
-                      const __nv_bfloat16* Hlo, double* partial, int* status_dev, cudaStream_t st) {
-  CUtensorMap ta, tb0, tb1;
-  int rc = make_tmap_bf16(&ta, D, static_cast<uint64_t>(in), static_cast<uint64_t>(m_total), static_cast<uint64_t>(in) * 2, 256);
+// Scorer contraction: for each stacked D (bf16 [rows][in]) the lower-triangle tiles of D^T D are
+// formed like the Hessian's and dotted with the fp32 H in the epilogue;
+// partial[tile][half][warp] holds each epilogue warp's share of sum(H .* D^T D).
+int gram_launch(const __nv_bfloat16* D0, const __nv_bfloat16* D1, int64_t rows, int64_t in, const float* H,
+                double* partial, int* status_dev, cudaStream_t st) {
+  CUtensorMap t0, t1;
+  int rc = make_tmap_bf16(&t0, D0, static_cast<uint64_t>(in), static_cast<uint64_t>(rows), static_cast<uint64_t>(in) * 2, kKT);
   if (rc != ADADIM_OK) return rc;
-  rc = make_tmap_bf16(&tb0, Hhi, static_cast<uint64_t>(in), static_cast<uint64_t>(in), static_cast<uint64_t>(in) * 2, 256);
-  if (rc != ADADIM_OK) return rc;
-  rc = make_tmap_bf16(&tb1, Hlo, static_cast<uint64_t>(in), static_cast<uint64_t>(in), static_cast<uint64_t>(in) * 2, 256);
+  rc = make_tmap_bf16(&t1, D1 != nullptr ? D1 : D0, static_cast<uint64_t>(in), static_cast<uint64_t>(rows),
+                      static_cast<uint64_t>(in) * 2, kKT);
   if (rc != ADADIM_OK) return rc;
   TcParams p = {};
-  p.tiles_n = static_cast<int>((in + 255) / 256);
-  p.num_tiles = static_cast<int>((m_total + 255) / 256) * p.tiles_n;
-  p.num_k = static_cast<int>((in + kKT - 1) / kKT);
+  const int nblk = static_cast<int>((in + 255) / 256);
+  p.tiles_per_dim = nblk * (nblk + 1) / 2;
+  p.num_tiles = p.tiles_per_dim * (D1 != nullptr ? 2 : 1);
+  p.num_k = static_cast<int>((rows + kKT - 1) / kKT);
   p.k_chunk = p.num_k;
   p.status_dev = status_dev;
-  p.D = D;
+  p.H = const_cast<float*>(H);        // read only in this mode
   p.in = in;
-  p.m_total = m_total;
   p.partial = partial;
-  return tc_launch<Mode::kScore>(ta, tb0, tb1, p, st);
+  return tc_launch<Mode::kGram>(t0, t1, t0, p, st);
 }
 
-int score_tiles(int64_t m_total, int64_t in) {
-  return static_cast<int>((m_total + 255) / 256) * static_cast<int>((in + 255) / 256);
+int gram_tiles(int64_t in) {
+  const int nblk = static_cast<int>((in + 255) / 256);
+  return nblk * (nblk + 1) / 2;
 }
 
 }  // namespace adadim

@@ -40,7 +40,7 @@ def test_workspace_sizes_grow_with_the_problem(lib):
     g1, g2 = f(1, 256, 512, 3, 128), f(1, 4096, 4096, 3, 128)
     s1, s2 = f(2, 256, 512, 3, 128), f(2, 4096, 4096, 3, 128)
     assert 0 < g1 < g2 and 0 < s1 < s2
-    assert s2 >= 2 * 4096 * 4096 * 2 + 2 * 4096 * 4096 * 2          # D for two dims + H in two bf16 parts
+    assert s2 >= 2 * 4096 * 4096 * 2                                # W - Q in bf16 for two dimensions
     assert f(3, 0, 4096, 0, 0) >= 4096 * 4096 * 8
 
 

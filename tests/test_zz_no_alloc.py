@@ -28,7 +28,7 @@ def _layer(out, inp, seed, bits, group):
 
 def test_static_scratch_matches_workspace_version_on_two_calls_in_a_row():
     assert B.static_scratch_bytes() == 16 << 20
-    cases = [(1024, 1024, 7101, 3, 128), (384, 512, 7201, 4, 64)]      # the first takes half of the array
+    cases = [(1024, 1024, 7101, 3, 128), (384, 512, 7201, 4, 64)]      # the first takes a quarter of the array
     layers = [_layer(*c) for c in cases]
     refs = []
     for (out, inp, _, bits, group), (W, H, q_oc, q_ic) in zip(cases, layers):
