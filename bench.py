@@ -106,7 +106,7 @@ def launches_per_step(out: int, inp: int) -> int:
     gptq = 1 + 1 + blocks + (blocks - 1) + 1           # init, U slicing, block kernels, trailing kernels, loss
     hessian = 2 if inp > 256 else 1
     rtn = 1
-    score = 2 + 1 + 1                                  # two difference kernels, Gram product, finalize
+    score = 1 + 1 + 1                                  # difference kernel, Gram product, finalize
     return hessian + rtn + score + factor + gptq + score
 
 

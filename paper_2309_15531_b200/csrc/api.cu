@@ -39,7 +39,7 @@ int check_quant_params(int bits, int group) {
 
 int check_qtensor(const adadim_qtensor* q) {
   if (q == nullptr || q->codes == nullptr || q->scales == nullptr || q->zeros == nullptr) return ADADIM_ERR_NULL;
-  if (!aligned16(q->codes)) return ADADIM_ERR_ALIGN;
+  if (!aligned16(q->codes) || !aligned16(q->scales) || !aligned16(q->zeros)) return ADADIM_ERR_ALIGN;
   return ADADIM_OK;
 }
 

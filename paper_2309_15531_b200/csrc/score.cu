@@ -17,50 +17,59 @@ int gram_tiles(int64_t in);
 
 namespace {
 
-// One thread dequantizes 32 consecutive codes of one row (BITS words) and writes W - Q as bf16.
+// W - Q as bf16 for one or both quantized tensors, from one read of W.  One thread handles
+// eight consecutive weights of a row (one 16-byte load and one 16-byte store per output), so
+// neighbouring threads touch neighbouring memory.  qa/Da are the per-OC tensor and its output,
+// qb/Db the per-IC ones; a null codes pointer skips that side.
 template <typename T, int BITS>
 __global__ void __launch_bounds__(256)
-diff_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int group, bool is_ic,
-            adadim_qtensor q, __nv_bfloat16* __restrict__ D) {
-  const int64_t chunks = in / 32;
+diff_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int group,
+            adadim_qtensor qa, __nv_bfloat16* __restrict__ Da, adadim_qtensor qb, __nv_bfloat16* __restrict__ Db) {
+  const int64_t vecs = in / 8;
   const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (t >= out * chunks) return;
-  const int64_t row = t / chunks, col0 = (t % chunks) * 32;
-  const uint32_t* src = q.codes + row * (in * BITS / 32) + col0 * BITS / 32;
-  uint32_t wds[BITS + 1];
+  if (t >= out * vecs) return;
+  const int64_t row = t / vecs, col0 = (t % vecs) * 8;
+  float w[8];
+  load8(W + row * ldw + col0, w);
+  // the eight codes start at bit col0*BITS of the row's stream: at most two words
+  const int64_t bit0 = col0 * BITS;
+  const int64_t word0 = row * (in * BITS / 32) + (bit0 >> 5);
+  const int sh0 = static_cast<int>(bit0 & 31);
+  const bool two = sh0 + 8 * BITS > 32;
 #pragma unroll
-  for (int k = 0; k < BITS; ++k) wds[k] = src[k];
-  wds[BITS] = 0;
-  float s_oc = 0.f, z_oc = 0.f;
-  if (!is_ic) {
-    int64_t idx = row * (in / group) + col0 / group;        // group >= 32: one group per chunk
-    s_oc = __half2float(__ushort_as_half(q.scales[idx]));
-    z_oc = __half2float(__ushort_as_half(q.zeros[idx]));
-  }
-  const uint16_t* sc = q.scales + (row / group) * in + col0;
-  const uint16_t* zr = q.zeros + (row / group) * in + col0;
+  for (int side = 0; side < 2; ++side) {
+    const adadim_qtensor& q = side == 0 ? qa : qb;
+    if (q.codes == nullptr) continue;
+    uint64_t bitsv = q.codes[word0];
+    if (two) bitsv |= static_cast<uint64_t>(q.codes[word0 + 1]) << 32;
+    bitsv >>= sh0;
+    float s[8], z[8];
+    if (side == 0) {
+      const int64_t idx = row * (in / group) + col0 / group;      // group >= 32: one group per vector
+      const float s0 = __half2float(__ushort_as_half(q.scales[idx]));
+      const float z0 = __half2float(__ushort_as_half(q.zeros[idx]));
 #pragma unroll
-  for (int v8 = 0; v8 < 4; ++v8) {
-    float w[8];
-    load8(W + row * ldw + col0 + v8 * 8, w);
+      for (int k = 0; k < 8; ++k) { s[k] = s0; z[k] = z0; }
+    } else {
+      const uint4 sv = *reinterpret_cast<const uint4*>(q.scales + (row / group) * in + col0);
+      const uint4 zv = *reinterpret_cast<const uint4*>(q.zeros + (row / group) * in + col0);
+      const __half2* sh = reinterpret_cast<const __half2*>(&sv);
+      const __half2* zh = reinterpret_cast<const __half2*>(&zv);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float2 a = __half22float2(sh[k]), b = __half22float2(zh[k]);
+        s[2 * k] = a.x; s[2 * k + 1] = a.y; z[2 * k] = b.x; z[2 * k + 1] = b.y;
+      }
+    }
     __nv_bfloat162 o[4];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const int kk = v8 * 8 + k;
-      const int bit = kk * BITS, wi = bit >> 5, sh = bit & 31;
-      uint32_t c = wds[wi] >> sh;
-      if (sh + BITS > 32) c |= wds[wi + 1] << (32 - sh);
-      c &= (1u << BITS) - 1u;
-      float s = s_oc, z = z_oc;
-      if (is_ic) {
-        s = __half2float(__ushort_as_half(sc[kk]));
-        z = __half2float(__ushort_as_half(zr[kk]));
-      }
-      float qv = __fmul_rn(s, static_cast<float>(c) - z);   // exact: 11-bit scale times a small integer
-      float d = __fsub_rn(w[k], qv);
+      const uint32_t c = static_cast<uint32_t>(bitsv >> (k * BITS)) & ((1u << BITS) - 1u);
+      const float qv = __fmul_rn(s[k], static_cast<float>(c) - z[k]);   // exact: 11-bit scale times a small integer
+      const float d = __fsub_rn(w[k], qv);
       if (k & 1) o[k >> 1].y = __float2bfloat16_rn(d); else o[k >> 1].x = __float2bfloat16_rn(d);
     }
-    *reinterpret_cast<uint4*>(D + row * in + col0 + v8 * 8) = *reinterpret_cast<uint4*>(o);
+    *reinterpret_cast<uint4*>((side == 0 ? Da : Db) + row * in + col0) = *reinterpret_cast<uint4*>(o);
   }
 }
 
@@ -102,12 +111,12 @@ finalize_kernel(const double* __restrict__ partial, int num_tiles, int tiles_fir
 }
 
 template <typename T>
-void diff_launch(const T* W, int64_t out, int64_t in, int64_t ldw, int bits, int group, bool is_ic,
-                 const adadim_qtensor& q, __nv_bfloat16* D, cudaStream_t st) {
-  int64_t n = out * (in / 32);
-  unsigned blocks = static_cast<unsigned>((n + 255) / 256);
-  if (bits == 3) diff_kernel<T, 3><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, is_ic, q, D);
-  else diff_kernel<T, 4><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, is_ic, q, D);
+void diff_launch(const T* W, int64_t out, int64_t in, int64_t ldw, int bits, int group, const adadim_qtensor& qa,
+                 __nv_bfloat16* Da, const adadim_qtensor& qb, __nv_bfloat16* Db, cudaStream_t st) {
+  const int64_t n = out * (in / 8);
+  const unsigned blocks = static_cast<unsigned>((n + 255) / 256);
+  if (bits == 3) diff_kernel<T, 3><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
+  else diff_kernel<T, 4><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
 }
 
 struct ScoreLayout {
@@ -134,17 +143,14 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
   __nv_bfloat16* D = reinterpret_cast<__nv_bfloat16*>(ws + L.d_off);
   double* partial = reinterpret_cast<double*>(ws + L.part_off);
 
-  const adadim_qtensor* qs[2] = {q_oc, q_ic};
   const int first_dim = q_oc != nullptr ? ADADIM_DIM_OC : ADADIM_DIM_IC;
   const bool have_second = q_oc != nullptr && q_ic != nullptr;
-  int64_t rows = 0;
-  for (int d = 0; d < 2; ++d) {
-    if (qs[d] == nullptr) continue;
-    __nv_bfloat16* dst = D + rows * in;
-    if (wdtype == ADADIM_F16) diff_launch(static_cast<const __half*>(W), out, in, ldw, bits, group, d == 1, *qs[d], dst, st);
-    else diff_launch(static_cast<const float*>(W), out, in, ldw, bits, group, d == 1, *qs[d], dst, st);
-    rows += out;
-  }
+  const adadim_qtensor none = {nullptr, nullptr, nullptr};
+  const adadim_qtensor qa = q_oc != nullptr ? *q_oc : none, qb = q_ic != nullptr ? *q_ic : none;
+  __nv_bfloat16* Da = D;                                        // first scored dimension first
+  __nv_bfloat16* Db = q_oc != nullptr ? D + out * in : D;
+  if (wdtype == ADADIM_F16) diff_launch(static_cast<const __half*>(W), out, in, ldw, bits, group, qa, Da, qb, Db, st);
+  else diff_launch(static_cast<const float*>(W), out, in, ldw, bits, group, qa, Da, qb, Db, st);
   if (cudaGetLastError() != cudaSuccess) return ADADIM_ERR_CUDA;
   int rc = gram_launch(D, have_second ? D + out * in : nullptr, out, in, H, partial, status_dev, st);
   if (rc != ADADIM_OK) return rc;

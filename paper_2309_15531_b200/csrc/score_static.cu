@@ -69,7 +69,7 @@ int adadim_score_select_static(const void* W, int wdtype, int64_t out, int64_t i
   for (int d = 0; d < 2; ++d) {
     if (qs[d] == nullptr) continue;
     if (qs[d]->codes == nullptr || qs[d]->scales == nullptr || qs[d]->zeros == nullptr) return ADADIM_ERR_NULL;
-    if (!aligned16(qs[d]->codes)) return ADADIM_ERR_ALIGN;
+    if (!aligned16(qs[d]->codes) || !aligned16(qs[d]->scales) || !aligned16(qs[d]->zeros)) return ADADIM_ERR_ALIGN;
     if ((d == 0 ? in : out) % group != 0) return ADADIM_ERR_SHAPE;
   }
   // the size limit: the layer's scoring workspace must fit the built-in array
