@@ -126,7 +126,8 @@ __device__ __forceinline__ void product128(const double* __restrict__ A, int64_t
     if (more) fetch(k0 + kBK);
 #pragma unroll
     for (int kk = 0; kk < kBK; ++kk) {
-      double a[8], b[8];
+      __align__(16) double a[8];
+      __align__(16) double b[8];
       *reinterpret_cast<double2*>(a + 0) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4]);
       *reinterpret_cast<double2*>(a + 2) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4 + 2]);
       *reinterpret_cast<double2*>(a + 4) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4]);

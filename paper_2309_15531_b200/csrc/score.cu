@@ -61,7 +61,7 @@ diff_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int g
         s[2 * k] = a.x; s[2 * k + 1] = a.y; z[2 * k] = b.x; z[2 * k + 1] = b.y;
       }
     }
-    __nv_bfloat162 o[4];
+    __align__(16) __nv_bfloat162 o[4];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const uint32_t c = static_cast<uint32_t>(bitsv >> (k * BITS)) & ((1u << BITS) - 1u);
