@@ -13,6 +13,24 @@ namespace {
 constexpr int kThreads = 256;       // 16 threads across a tile row (8 columns each) x 16 rows
 constexpr int kPasses = 8;          // 16 rows per pass
 
+// Eight codes of one row segment from the correctly rounded quotients: adding 1.5 * 2^23 leaves
+// rint(q) in the low mantissa bits; code = clamp(bits - bias, 0, maxq) with bias = magic - z is
+// one integer add-min-relu; the codes are packed by multiply-add.  |q| stays far below 2^22
+// here because every weight lies inside its own group's range.
+template <int BITS>
+__device__ __forceinline__ uint32_t pack8(const float (&w)[8], const float (&s)[8], const float (&r)[8],
+                                          const int (&nbias)[8]) {
+  constexpr int maxq = (1 << BITS) - 1;
+  uint32_t acc = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const float t = __fadd_rn(quotient(w[k], s[k], r[k]), kRoundMagic);
+    const int c = __viaddmin_s32_relu(__float_as_int(t), nbias[k], maxq);
+    acc = static_cast<uint32_t>(c) * (1u << (BITS * k)) + acc;
+  }
+  return acc;
+}
+
 // Pack eight codes (column order) of `BITS` bits and hand back this thread's share of the
 // row's bitstream.  acc arrives as sum_k(tbits_k << BITS*k) - bias, i.e. the packed value.
 template <int BITS>
@@ -36,7 +54,6 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
   constexpr int NG = kTile / G;               // per-IC groups stacked in one tile
   constexpr int PPG = kPasses / NG;           // passes per such group
   constexpr int LANES_PER_OCG = G / 8;        // threads sharing one per-OC group
-  constexpr uint32_t kOnes = BITS == 3 ? 0x00249249u : 0x11111111u;   // sum_k 1 << BITS*k
 
   __shared__ float s_mn[NG][8][kTile];
   __shared__ float s_mx[NG][8][kTile];
@@ -115,16 +132,15 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
   // ---- codes ------------------------------------------------------------------------------
 #pragma unroll
   for (int gi = 0; gi < NG; ++gi) {
-    float ic_s[8], ic_r[8], ic_z[8];
-    uint32_t ic_bias = 0;
+    float ic_s[8], ic_r[8];
+    int ic_nb[8];
     if (DO_IC) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         float s = s_s[gi][colvec * 8 + k];
-        ic_z[k] = s_z[gi][colvec * 8 + k];
         ic_r[k] = s == 0.0f ? 0.0f : __frcp_rn(s);
         ic_s[k] = s == 0.0f ? 1.0f : s;
-        ic_bias += static_cast<uint32_t>(kRoundMagicBits - static_cast<int>(ic_z[k])) << (BITS * k);
+        ic_nb[k] = static_cast<int>(s_z[gi][colvec * 8 + k]) - kRoundMagicBits;
       }
     }
 #pragma unroll
@@ -147,26 +163,15 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
           qoc.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
           qoc.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
         }
-        uint32_t acc = 0;
-        const float zlo = kRoundMagic - gp.z, zhi = kRoundMagic + (maxq - gp.z);
+        float s8[8], r8[8];
+        int nb8[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          float t = __fadd_rn(quotient(w[p][k], gp.s, gp.rcp), kRoundMagic);
-          t = fminf(fmaxf(t, zlo), zhi);
-          acc += static_cast<uint32_t>(__float_as_int(t)) << (BITS * k);
-        }
-        acc -= static_cast<uint32_t>(kRoundMagicBits - static_cast<int>(gp.z)) * kOnes;
+        for (int k = 0; k < 8; ++k) { s8[k] = gp.s; r8[k] = gp.rcp; nb8[k] = static_cast<int>(gp.z) - kRoundMagicBits; }
+        const uint32_t acc = pack8<BITS>(w[p], s8, r8, nb8);
         store_codes<BITS>(acc, qoc.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
       }
       if (DO_IC) {
-        uint32_t acc = 0;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          float t = __fadd_rn(quotient(w[p][k], ic_s[k], ic_r[k]), kRoundMagic);
-          t = fminf(fmaxf(t, kRoundMagic - ic_z[k]), kRoundMagic + (maxq - ic_z[k]));
-          acc += static_cast<uint32_t>(__float_as_int(t)) << (BITS * k);
-        }
-        acc -= ic_bias;
+        const uint32_t acc = pack8<BITS>(w[p], ic_s, ic_r, ic_nb);
         store_codes<BITS>(acc, qic.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
       }
     }
