@@ -12,7 +12,7 @@
 //                   multiplied by the inverted diagonal block).  Panels are grouped four at a
 //                   time: inside a group only the group's own columns are updated after each
 //                   panel; the rest of the matrix gets one rank-256 update per group, on
-//                   128 x 128 tiles (high arithmetic intensity).
+//                   128 x 64 tiles.
 //   inverse       : recursive doubling.  inv([[A,0],[C,B]]) = [[A^-1,0],[-B^-1 C A^-1,B^-1]]:
 //                   level by level, adjacent inverted diagonal blocks are merged with two
 //                   batched triangular-aware matrix products, log2(n/64) levels in all.
@@ -73,90 +73,90 @@ __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64
   __shared__ double sa[16][kNB + 2];   \
   __shared__ double sb[16][kNB + 2];
 
-// ---- 128 x 128 output tile product, 256 threads, 8 x 8 outputs per thread ------------------
-// Output rows of a thread: ty*4 + {0..3} and 64 + ty*4 + {0..3}; columns likewise with tx.
-// Rows >= a_rows of A and columns >= b_cols of B are not read (treated as zero); both limits
-// are 64 or 128.  K is a multiple of 8.  Shared-memory slabs are double-buffered and the next
-// slab is fetched into registers while the current one is multiplied.
-constexpr int kT = 128, kBK = 8, kLd = kT + 4;
-struct Tile128Smem {
-  double a[2][kBK][kLd];
-  double b[2][kBK][kLd];
+// ---- 128 x 64 output tile product, 256 threads, 8 x 4 outputs per thread -------------------
+// Output rows of a thread: ty*4 + {0..3} and 64 + ty*4 + {0..3}; columns tx*4 + {0..3}.
+// Rows >= a_rows (64 or 128) of A are not read (treated as zero).  K is a multiple of 8.
+// Shared-memory slabs are double-buffered; the slab after the next one is already on its way
+// from global memory into registers while the current one is multiplied, and two CTAs share an
+// SM, so global latency is covered.
+constexpr int kT = 128, kTN = 64, kBK = 8;
+struct TileSmem {
+  double a[2][kBK][kT + 4];
+  double b[2][kBK][kTN + 4];
 };
 
 template <bool B_T>
-__device__ __forceinline__ void product128(const double* __restrict__ A, int64_t lda, int a_rows,
-                                           const double* __restrict__ B, int64_t ldb, int b_cols, int K,
-                                           double (&acc)[8][8], Tile128Smem& sm) {
+__device__ __forceinline__ void product_tile(const double* __restrict__ A, int64_t lda, int a_rows,
+                                             const double* __restrict__ B, int64_t ldb, int K,
+                                             double (&acc)[8][4], TileSmem& sm) {
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int ar = tid >> 1, akq = (tid & 1) * 4;                 // A loader: row, first k of four
-  const int bkk = tid >> 5, bnq = (tid & 31) * 4;               // B loader (not transposed): k row, first col
+  const int br = tid >> 2, bkq = (tid & 3) * 2;                 // B loader (transposed): column, first k of two
+  const int bkk = tid >> 5, bnq = (tid & 31) * 2;               // B loader (not transposed): k row, first col of two
   const bool a_ok = ar < a_rows;
-  const bool b_ok = B_T ? (ar < b_cols) : (bnq < b_cols);
   const double* ap = A + static_cast<int64_t>(ar) * lda + akq;
-  const double* bp = B_T ? B + static_cast<int64_t>(ar) * ldb + akq : B + static_cast<int64_t>(bkk) * ldb + bnq;
+  const double* bp = B_T ? B + static_cast<int64_t>(br) * ldb + bkq : B + static_cast<int64_t>(bkk) * ldb + bnq;
   const int64_t bstep = B_T ? kBK : static_cast<int64_t>(kBK) * ldb;
-  double2 ra0, ra1, rb0, rb1;
   const double2 zero2 = make_double2(0.0, 0.0);
+  struct Slab { double2 a0, a1, b; };                           // one thread's share of a slab
+  Slab s0, s1;                                                  // two slabs in flight
 
-  auto fetch = [&](int k0) {
-    if (a_ok) { const double2* s = reinterpret_cast<const double2*>(ap + k0); ra0 = s[0]; ra1 = s[1]; }
-    else { ra0 = zero2; ra1 = zero2; }
-    if (b_ok) { const double2* s = reinterpret_cast<const double2*>(bp + (k0 / kBK) * bstep); rb0 = s[0]; rb1 = s[1]; }
-    else { rb0 = zero2; rb1 = zero2; }
+  auto fetch = [&](Slab& r, int k0) {
+    if (a_ok) { const double2* g = reinterpret_cast<const double2*>(ap + k0); r.a0 = g[0]; r.a1 = g[1]; }
+    else { r.a0 = zero2; r.a1 = zero2; }
+    r.b = *reinterpret_cast<const double2*>(bp + (k0 / kBK) * bstep);
   };
-  auto stash = [&](int buf) {
-    sm.a[buf][akq + 0][ar] = ra0.x; sm.a[buf][akq + 1][ar] = ra0.y;
-    sm.a[buf][akq + 2][ar] = ra1.x; sm.a[buf][akq + 3][ar] = ra1.y;
-    if (B_T) {
-      sm.b[buf][akq + 0][ar] = rb0.x; sm.b[buf][akq + 1][ar] = rb0.y;
-      sm.b[buf][akq + 2][ar] = rb1.x; sm.b[buf][akq + 3][ar] = rb1.y;
-    } else {
-      *reinterpret_cast<double2*>(&sm.b[buf][bkk][bnq]) = rb0;
-      *reinterpret_cast<double2*>(&sm.b[buf][bkk][bnq + 2]) = rb1;
-    }
+  auto stash = [&](const Slab& r, int buf) {
+    sm.a[buf][akq + 0][ar] = r.a0.x; sm.a[buf][akq + 1][ar] = r.a0.y;
+    sm.a[buf][akq + 2][ar] = r.a1.x; sm.a[buf][akq + 3][ar] = r.a1.y;
+    if (B_T) { sm.b[buf][bkq][br] = r.b.x; sm.b[buf][bkq + 1][br] = r.b.y; }
+    else *reinterpret_cast<double2*>(&sm.b[buf][bkk][bnq]) = r.b;
   };
-
-  fetch(0);
-  stash(0);
-  __syncthreads();
-  int buf = 0;
-  for (int k0 = 0; k0 < K; k0 += kBK) {
-    const bool more = k0 + kBK < K;
-    if (more) fetch(k0 + kBK);
+  auto multiply = [&](int buf) {
 #pragma unroll
     for (int kk = 0; kk < kBK; ++kk) {
       __align__(16) double a[8];
-      __align__(16) double b[8];
+      __align__(16) double b[4];
       *reinterpret_cast<double2*>(a + 0) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4]);
       *reinterpret_cast<double2*>(a + 2) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4 + 2]);
       *reinterpret_cast<double2*>(a + 4) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4]);
       *reinterpret_cast<double2*>(a + 6) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4 + 2]);
       *reinterpret_cast<double2*>(b + 0) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][tx * 4]);
       *reinterpret_cast<double2*>(b + 2) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][tx * 4 + 2]);
-      *reinterpret_cast<double2*>(b + 4) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][64 + tx * 4]);
-      *reinterpret_cast<double2*>(b + 6) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][64 + tx * 4 + 2]);
 #pragma unroll
       for (int m = 0; m < 8; ++m)
 #pragma unroll
-        for (int n = 0; n < 8; ++n) acc[m][n] = fma(a[m], b[n], acc[m][n]);
+        for (int n = 0; n < 4; ++n) acc[m][n] = fma(a[m], b[n], acc[m][n]);
     }
-    if (more) stash(buf ^ 1);
+  };
+
+  // slab i is multiplied from buffer i & 1 while slab i+1 moves from registers to the other
+  // buffer and slab i+2 starts its trip from global memory
+  const int nslab = K / kBK;
+  fetch(s0, 0);
+  if (nslab > 1) fetch(s1, kBK);
+  stash(s0, 0);
+  __syncthreads();
+  for (int i = 0; i < nslab; i += 2) {
+    if (i + 1 < nslab) stash(s1, 1);
+    if (i + 2 < nslab) fetch(s0, (i + 2) * kBK);
+    multiply(0);
     __syncthreads();
-    buf ^= 1;
+    if (i + 1 < nslab) {
+      if (i + 2 < nslab) stash(s0, 0);
+      if (i + 3 < nslab) fetch(s1, (i + 3) * kBK);
+      multiply(1);
+      __syncthreads();
+    }
   }
 }
 
-// Applies f(row, col4, values of 4 consecutive columns) to a thread's 8 x 8 outputs.
+// Applies f(row, first column, values of 4 consecutive columns) to a thread's 8 x 4 outputs.
 template <typename F>
-__device__ __forceinline__ void for_each_quad(double (&acc)[8][8], F f) {
+__device__ __forceinline__ void for_each_quad(double (&acc)[8][4], F f) {
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
-  for (int m = 0; m < 8; ++m) {
-    const int r = (m < 4 ? 0 : 64) + ty * 4 + (m & 3);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) f(r, h * 64 + tx * 4, &acc[m][h * 4]);
-  }
+  for (int m = 0; m < 8; ++m) f((m < 4 ? 0 : 64) + ty * 4 + (m & 3), tx * 4, &acc[m][0]);
 }
 
 // ---- set-up --------------------------------------------------------------------------------
@@ -360,25 +360,27 @@ group_update_kernel(double* __restrict__ A, int64_t n, int k) {
     for (int q = 0; q < 4; ++q) c[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + q] -= acc[m][q];
 }
 
-// Rank-`kw` update of everything right of a finished group:  for 128 x 128 tiles (ti >= tj) of
-// the region starting at row/column e:  A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T.
-// Diagonal tiles do not store their upper-right 64 x 64 quadrant (it must stay zero).
-__global__ void __launch_bounds__(256, 1)
+// Rank-`kw` update of everything right of a finished group:  for tiles of 128 rows x 64 columns on
+// or below the diagonal of the region starting at row/column e:
+//   A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T.
+// Row block ti meets column blocks 0 .. 2*ti+1.  The tile right of the diagonal 64-block (column
+// block 2*ti+1) only stores its lower 64 rows: the block above them must stay zero.
+__global__ void __launch_bounds__(256, 2)
 rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
-  __shared__ Tile128Smem sm;
-  int t = blockIdx.x;
-  int ti = static_cast<int>((sqrt(8.0 * t + 1.0) - 1.0) * 0.5);
-  while (ti * (ti + 1) / 2 > t) --ti;
-  while ((ti + 1) * (ti + 2) / 2 <= t) ++ti;
-  const int tj = t - ti * (ti + 1) / 2;
-  const int64_t ri = e + static_cast<int64_t>(ti) * kT, rj = e + static_cast<int64_t>(tj) * kT;
-  const int vr = static_cast<int>(mn64(kT, n - ri)), vc = static_cast<int>(mn64(kT, n - rj));
-  double acc[8][8] = {};
-  product128<true>(A + ri * n + j0, n, vr, A + rj * n + j0, n, vc, kw, acc, sm);
-  const bool diag = ti == tj;
+  __shared__ TileSmem sm;
+  const int t = blockIdx.x;
+  int ti = static_cast<int>((sqrt(4.0 * t + 1.0) - 1.0) * 0.5);
+  while (ti * (ti + 1) > t) --ti;
+  while ((ti + 1) * (ti + 2) <= t) ++ti;
+  const int cj = t - ti * (ti + 1);
+  const int64_t ri = e + static_cast<int64_t>(ti) * kT, rj = e + static_cast<int64_t>(cj) * kTN;
+  if (rj >= n) return;
+  const int vr = static_cast<int>(mn64(kT, n - ri));
+  double acc[8][4] = {};
+  product_tile<true>(A + ri * n + j0, n, vr, A + rj * n + j0, n, kw, acc, sm);
+  const int skip_rows = cj == 2 * ti + 1 ? 64 : 0;
   for_each_quad(acc, [&](int r, int c4, const double* v) {
-    if (r >= vr || c4 >= vc) return;
-    if (diag && r < 64 && c4 >= 64) return;
+    if (r >= vr || r < skip_rows) return;
     double2* p = reinterpret_cast<double2*>(A + (ri + r) * n + rj + c4);
     double2 u0 = p[0], u1 = p[1];
     u0.x -= v[0]; u0.y -= v[1]; u1.x -= v[2]; u1.y -= v[3];
@@ -430,19 +432,19 @@ merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T
     for (int q = 0; q < 4; ++q) dst[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + q] = -acc[m][q];
 }
 
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(256, 2)
 merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T) {      // s >= 128
-  __shared__ Tile128Smem sm;
-  const int tiles = static_cast<int>(s / kT);
+  __shared__ TileSmem sm;
+  const int ctiles = static_cast<int>(s / kTN);
   const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  const int r = blockIdx.x / tiles, c = blockIdx.x % tiles;
+  const int r = blockIdx.x / ctiles, c = blockIdx.x % ctiles;          // 128-row block, 64-column block
   const int64_t sB = mn64(s, n - b0);
   if (static_cast<int64_t>(r) * kT >= sB) return;
   const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
-  const int64_t m0 = static_cast<int64_t>(c) * kT;
-  double acc[8][8] = {};
-  product128<false>(A + (b0 + static_cast<int64_t>(r) * kT) * n + a0 + m0, n, vr, A + (a0 + m0) * n + a0 + m0, n, kT,
-                    static_cast<int>(s - m0), acc, sm);
+  const int64_t m0 = static_cast<int64_t>(c) * kTN;
+  double acc[8][4] = {};
+  product_tile<false>(A + (b0 + static_cast<int64_t>(r) * kT) * n + a0 + m0, n, vr, A + (a0 + m0) * n + a0 + m0, n,
+                      static_cast<int>(s - m0), acc, sm);
   double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kT * s + m0;
   for_each_quad(acc, [&](int rr, int c4, const double* v) {
     if (rr >= vr) return;
@@ -451,21 +453,21 @@ merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __rest
     p[1] = make_double2(v[2], v[3]);
   });
 }
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(256, 2)
 merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T) {      // s >= 128
-  __shared__ Tile128Smem sm;
-  const int tiles = static_cast<int>(s / kT);
+  __shared__ TileSmem sm;
+  const int ctiles = static_cast<int>(s / kTN);
   const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  const int r = blockIdx.x / tiles, c = blockIdx.x % tiles;
+  const int r = blockIdx.x / ctiles, c = blockIdx.x % ctiles;
   const int64_t sB = mn64(s, n - b0);
   if (static_cast<int64_t>(r) * kT >= sB) return;
   const int64_t row0 = b0 + static_cast<int64_t>(r) * kT;
   const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
   const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kT, sB));
-  double acc[8][8] = {};
-  product128<false>(A + row0 * n + b0, n, vr, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kT, s,
-                    kT, K, acc, sm);
-  double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kT;
+  double acc[8][4] = {};
+  product_tile<false>(A + row0 * n + b0, n, vr, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kTN,
+                      s, K, acc, sm);
+  double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kTN;
   for_each_quad(acc, [&](int rr, int c4, const double* v) {
     if (rr >= vr) return;
     double2* p = reinterpret_cast<double2*>(dst + static_cast<int64_t>(rr) * n + c4);
@@ -524,7 +526,7 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
     const int64_t e = static_cast<int64_t>(g1) * kNB;
     if (e < n) {
       const int nt = static_cast<int>((n - e + kT - 1) / kT);
-      rank_update_kernel<<<nt * (nt + 1) / 2, 256, 0, st>>>(A, n, e, static_cast<int64_t>(g0) * kNB, (g1 - g0) * kNB);
+      rank_update_kernel<<<nt * (nt + 1), 256, 0, st>>>(A, n, e, static_cast<int64_t>(g0) * kNB, (g1 - g0) * kNB);
     }
   }
   seed_kernel<<<nb, 256, 0, st>>>(A, n, dinv);
@@ -535,7 +537,7 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
   }
   for (int64_t s = 2 * kNB; s < n; s *= 2) {
     const unsigned pairs = static_cast<unsigned>((n + 2 * s - 1) / (2 * s));
-    const unsigned tiles = static_cast<unsigned>((s / kT) * (s / kT));
+    const unsigned tiles = static_cast<unsigned>((s / kT) * (s / kTN));
     merge1_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
     merge2_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
   }
