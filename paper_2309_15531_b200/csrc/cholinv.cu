@@ -197,132 +197,72 @@ build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ 
 }
 
 // ---- factorization -------------------------------------------------------------------------
-// Cholesky of a 32 x 32 block by one warp, rows in registers (lane r holds row r; entries right
-// of the diagonal are don't-cares).  Right-looking: the pivot and the scaled column travel by
-// shuffles, so there is no block-wide barrier in the sequential part.  rdiag[j] = 1 / L[j][j].
-__device__ __forceinline__ void chol32_warp(double (&a)[32], double* rdiag, int* status_dev) {
-  const int lane = threadIdx.x & 31;
-#pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    double d = __shfl_sync(0xffffffffu, a[j], j);
-    if (!(d > 0.0)) {
-      if (lane == 0) report(status_dev, ADADIM_ERR_NOT_PD);
-      d = 1.0;
-    }
-    const double r = rsqrt(d);
-    const double l = a[j] * r;
-    a[j] = l;
-    if (lane == 0) rdiag[j] = r;
-#pragma unroll
-    for (int c = j + 1; c < 32; ++c) a[c] = fma(-l, __shfl_sync(0xffffffffu, l, c), a[c]);
-  }
-}
-
-// Inverse of a 32 x 32 lower-triangular block by one warp: lane c solves column c by forward
-// substitution; Ls is the block in shared memory (pitch ld), x[r] = X[r][c].
-__device__ __forceinline__ void trinv32_warp(const double* Ls, int ld, const double* rdiag, double (&x)[32]) {
-  const int c = threadIdx.x & 31;
-#pragma unroll
-  for (int r = 0; r < 32; ++r) {
-    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-#pragma unroll
-    for (int m = 0; m < r; ++m) {
-      const double l = Ls[r * ld + m];
-      if ((m & 3) == 0) s0 = fma(l, x[m], s0);
-      else if ((m & 3) == 1) s1 = fma(l, x[m], s1);
-      else if ((m & 3) == 2) s2 = fma(l, x[m], s2);
-      else s3 = fma(l, x[m], s3);
-    }
-    x[r] = ((r == c ? 1.0 : 0.0) - ((s0 + s1) + (s2 + s3))) * rdiag[r];
-  }
-}
-
-// Diagonal block k: in-place Cholesky of the 64 x 64 block and its triangular inverse -> dinv[k],
-// as a 2 x 2 arrangement of 32 x 32 blocks: factor and invert A11 on one warp, L21 = A21 X11^T and
-// A22 -= L21 L21^T on the whole CTA, factor and invert A22, X21 = -X22 (L21 X11).
+// Diagonal block k: in-place Cholesky of the 64 x 64 block and its triangular inverse -> dinv[k].
+// Column by column (left-looking): four threads share a row's dot product; the pivot's
+// reciprocal square root scales the column.  The inverse is a forward substitution with four
+// threads per column, the column's entries spread over their registers.
 __global__ void __launch_bounds__(256)
-potrf_kernel(double* __restrict__ A, int64_t n, int k, double* dinv, int* status_dev) {
-  constexpr int LD = kNB + 1;
-  __shared__ double L[kNB * LD];
-  __shared__ double Ts[32 * 33];
-  __shared__ double rdiag[kNB];
+potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv, int* status_dev) {
+  __shared__ double L[kNB][kNB + 1];
+  __shared__ double col[kNB];
+  __shared__ double rdiag[kNB];          // 1 / L[j][j]
   double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
-  double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;      // X, row-major 64 x 64
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  for (int e = tid; e < kNB * kNB; e += 256) L[(e >> 6) * LD + (e & 63)] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
+  for (int e = threadIdx.x; e < kNB * kNB; e += 256) L[e >> 6][e & 63] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
   __syncthreads();
-
-  // each of the two 32-blocks: factor, write back, invert, store the inverse in dk
-  auto diag_block = [&](int o) {
-    double a[32];
-#pragma unroll
-    for (int c = 0; c < 32; ++c) a[c] = L[(o + lane) * LD + o + c];
-    chol32_warp(a, rdiag + o, status_dev);
-#pragma unroll
-    for (int c = 0; c < 32; ++c) L[(o + lane) * LD + o + c] = c <= lane ? a[c] : 0.0;
-    __syncwarp();
-    double x[32];
-    trinv32_warp(L + o * LD + o, LD, rdiag + o, x);
-#pragma unroll
-    for (int r = 0; r < 32; ++r) dk[(o + r) * kNB + o + lane] = r < lane ? 0.0 : x[r];
-  };
-  // 32 x 32 x 32 product on the CTA: thread -> row i, four consecutive columns j0..j0+3
-  const int pi = tid >> 3, pj = (tid & 7) * 4;
-
-  if (warp == 0) diag_block(0);
-  __syncthreads();
-  {   // L21 = A21 * X11^T
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int kk = 0; kk < 32; ++kk) {
-      const double av = L[(32 + pi) * LD + kk];
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) acc[jj] = fma(av, dk[(pj + jj) * kNB + kk], acc[jj]);
+  const int row = threadIdx.x >> 2, q = threadIdx.x & 3;
+#pragma unroll 1
+  for (int j = 0; j < kNB; ++j) {
+    double s0 = 0.0, s1 = 0.0;
+    if (row >= j) {
+      int m = q;
+      for (; m + 4 < j; m += 8) {                      // entries m = q, q+4, ... < j of the two rows
+        s0 = fma(L[row][m], L[j][m], s0);
+        s1 = fma(L[row][m + 4], L[j][m + 4], s1);
+      }
+      if (m < j) s0 = fma(L[row][m], L[j][m], s0);
     }
+    double sum = s0 + s1;
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+    if (q == 0 && row >= j) col[row] = L[row][j] - sum;
     __syncthreads();
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) L[(32 + pi) * LD + pj + jj] = acc[jj];
-  }
-  __syncthreads();
-  {   // A22 -= L21 * L21^T
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int kk = 0; kk < 32; ++kk) {
-      const double av = L[(32 + pi) * LD + kk];
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) acc[jj] = fma(av, L[(32 + pj + jj) * LD + kk], acc[jj]);
+    double piv = col[j];
+    if (!(piv > 0.0)) {
+      if (threadIdx.x == 0) report(status_dev, ADADIM_ERR_NOT_PD);
+      piv = 1.0;
     }
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) L[(32 + pi) * LD + 32 + pj + jj] -= acc[jj];
+    const double r = rsqrt(piv);
+    if (q == 0 && row >= j) L[row][j] = col[row] * r;
+    if (threadIdx.x == 0) rdiag[j] = r;
+    __syncthreads();
   }
-  __syncthreads();
-  if (warp == 0) diag_block(32);
-  __syncthreads();
-  {   // T = L21 * X11
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int kk = 0; kk < 32; ++kk) {
-      const double av = L[(32 + pi) * LD + kk];
+  // X = L^-1: thread (c, q) keeps X[m][c] for m = 4t + q in x[t]
+  {
+    const int c = row;
+    double x[kNB / 4];
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) acc[jj] = fma(av, dk[kk * kNB + pj + jj], acc[jj]);
-    }
+    for (int t = 0; t < kNB / 4; ++t) x[t] = 0.0;
+    double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) Ts[pi * 33 + pj + jj] = acc[jj];
-  }
-  __syncthreads();
-  {   // X21 = -X22 * T ;  the upper-right block of X is zero
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int kk = 0; kk < 32; ++kk) {
-      const double av = dk[(32 + pi) * kNB + 32 + kk];
+    for (int r = 0; r < kNB; ++r) {
+      double s0 = 0.0, s1 = 0.0;
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) acc[jj] = fma(av, Ts[kk * 33 + pj + jj], acc[jj]);
-    }
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      dk[(32 + pi) * kNB + pj + jj] = -acc[jj];
-      dk[pi * kNB + 32 + pj + jj] = 0.0;
+      for (int t = 0; t < (r + 3) / 4; ++t) {            // entries m = 4t + q < r
+        const int m = 4 * t + q;
+        const double l = m < r ? L[r][m] : 0.0;
+        if (t & 1) s1 = fma(l, x[t], s1); else s0 = fma(l, x[t], s0);
+      }
+      double sum = s0 + s1;
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      const double xr = ((r == c ? 1.0 : 0.0) - sum) * rdiag[r];
+      if (q == (r & 3)) x[r >> 2] = xr;
+      if (q == 0) dk[r * kNB + c] = r < c ? 0.0 : xr;
     }
   }
-  for (int e = tid; e < kNB * kNB; e += 256) {
+  for (int e = threadIdx.x; e < kNB * kNB; e += 256) {
     int r = e >> 6, c = e & 63;
-    blk[static_cast<int64_t>(r) * n + c] = r >= c ? L[r * LD + c] : 0.0;
+    blk[static_cast<int64_t>(r) * n + c] = r >= c ? L[r][c] : 0.0;
   }
 }
 

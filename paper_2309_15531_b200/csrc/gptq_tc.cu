@@ -23,7 +23,7 @@
 namespace adadim {
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                      // TMA warp, MMA warp, eight epilogue warps
 constexpr uint32_t kAPiece = 128 * 64 * 2;          // one Err piece, one 64-deep half of K: 16 KB
 constexpr uint32_t kABytes = 6 * kAPiece;           // 3 pieces x 2 halves
 constexpr int kTileN = 128;
@@ -70,7 +70,7 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
   if (threadIdx.x == 0) {
     ptx::mbar_init(a_full, 1);
     for (int s = 0; s < kBStages; ++s) { ptx::mbar_init(&b_full[s], 1); ptx::mbar_init(&b_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { ptx::mbar_init(&acc_full[s], 1); ptx::mbar_init(&acc_empty[s], 4); }
+    for (int s = 0; s < 2; ++s) { ptx::mbar_init(&acc_full[s], 1); ptx::mbar_init(&acc_empty[s], 8); }
     ptx::mbar_init(drain, 1);
     *dead = 0;
     ptx::fence_mbar_init();
@@ -165,23 +165,24 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
       }
     }
   } else {
-    const int q = warp & 3;
+    // two warps per TMEM lane quadrant, each taking one 64-column half of every tile
+    const int q = warp & 3, half = (warp - 2) >> 2;
     uint32_t acc_phase[2] = {0, 0};
-    float* wrow = p.Wc + (static_cast<int64_t>(mrow) + q * 32 + lane) * p.in;
+    float* wrow = p.Wc + (static_cast<int64_t>(mrow) + q * 32 + lane) * p.in + half * 64;
     for (int t = t0; t < t1; ++t) {
       const int buf = (t - t0) & 1;
       // The tile's slice of W does not depend on the MMAs: fetch it while they run.
       // (in % 128 == 0 and c0 % 128 == 0, so every tile lies wholly inside the matrix.)
       float4* w4 = reinterpret_cast<float4*>(wrow + p.c0 + static_cast<int64_t>(t) * kTileN);
-      float4 w[kTileN / 4];
+      float4 w[16];
 #pragma unroll
-      for (int k = 0; k < kTileN / 4; ++k) w[k] = w4[k];
+      for (int k = 0; k < 16; ++k) w[k] = w4[k];
       if (!ptx::mbar_wait(&acc_full[buf], acc_phase[buf], dead, p.status_dev)) break;
       ptx::tc_fence_after_sync();
 #pragma unroll
-      for (int c = 0; c < kTileN / 32; ++c) {
+      for (int c = 0; c < 2; ++c) {
         float v[32], v2[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + c * 32;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + half * 64 + c * 32;
         ptx::tmem_ld32(taddr, v);
         ptx::tmem_ld32(taddr + kTileN, v2);
 #pragma unroll
