@@ -138,4 +138,18 @@ def test_full_size_q_proj_sampled_slabs():
     wspec, xspec = wl["layers"]["q_proj"]
     W = I.make_weight(wspec, "cuda")
     X = I.make_calib(xspec, "cuda")
-    _gptq_case(W, X, 3, 128, rows=slice(1280, 1536))
+    out = _gptq_case(W, X, 3, 128, rows=slice(1280, 1536))
+    # internal consistency of the library's own result over the whole layer: the reported loss
+    # 1/2 sum(e^2) equals 1/2 trace(D Hd D^T) for its own D = W - Q (the products in fp64 by torch)
+    Hn = _hessian_f32(X)
+    Hd, _ = O.damped_hessian(Hn.astype(np.float64), 0.01)
+    Hd_t = torch.as_tensor(Hd, device="cuda")
+    loss = torch.zeros(2, dtype=torch.float64, device="cuda")
+    q_oc, q_ic = B.quantize_gptq(W, torch.as_tensor(Hn, device="cuda"), 3, 128, B.DIM_BOTH, 0.01, loss=loss)
+    Wn = to_np(W).astype(np.float32)
+    for k, (name, q) in enumerate((("oc", q_oc), ("ic", q_ic))):
+        codes, s, z = q_to_np(q)
+        D = torch.as_tensor(Wn.astype(np.float64) - O.dequantize(codes, s, z, 128, name).astype(np.float64), device="cuda")
+        tr = 0.5 * float(((D @ Hd_t) * D).sum().item())
+        print(f"gptq {name}: loss {loss[k].item():.6e}  1/2 trace(D Hd D^T) {tr:.6e}")
+        assert loss[k].item() == pytest.approx(tr, rel=1e-3)
