@@ -178,6 +178,260 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
   }
 }
 
+// ---- fp16 weights --------------------------------------------------------------------------
+// The same tile, kept in registers as it was loaded (f16x2 words) and widened to fp32 only where
+// the codes are formed.  Differences from the general kernel above, all exact:
+//  * minima and maxima are taken on f16x2 words (an fp16 minimum is exact);
+//  * the per-OC statistics of the eight passes are reduced across the lanes of a group by a
+//    reduce-scatter, so each lane ends up owning one (row, group), computes its parameters once
+//    and hands reciprocal and zero point to the others by shuffle when the codes are formed;
+//  * rint(w / s) for fp16 w and s needs no correctly rounded quotient.  Write w = a 2^x and
+//    s = b 2^y with integers |a|, b < 2^11: w/s - (m + 1/2) is either 0 or at least 2^-13 in
+//    magnitude for every integer m (its numerator is a non-zero integer over a denominator of
+//    at most 2^13 whenever |w/s| >= 1/2).  p = w * rcp(s) is within 2^-20 of w/s for |w/s| <= 16.
+//    fma(w, rcp, 192) rounds p to a multiple of 2^-16: an exact tie comes out as exactly m + 1/2,
+//    everything else stays on its side of every m + 1/2.  Adding 1.5 * 2^23 - 192 then rounds
+//    that to an integer, ties to even, which is rint of the correctly rounded quotient.
+constexpr float kSnapMagic = 192.0f;                     // 1.5 * 2^7: ulp 2^-16 in [128, 256)
+constexpr float kSnapToInt = 12582912.0f - 192.0f;       // exact in binary32
+
+__device__ __forceinline__ uint32_t min_h2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t max_h2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ float lo_h2(uint32_t v) { return __half2float(__ushort_as_half(static_cast<unsigned short>(v & 0xffffu))); }
+__device__ __forceinline__ float hi_h2(uint32_t v) { return __half2float(__ushort_as_half(static_cast<unsigned short>(v >> 16))); }
+
+// volatile keeps the widening beside its use: only the packed tile stays live across the passes.
+__device__ __forceinline__ void widen_h2(uint32_t v, float& a, float& b) {
+  asm volatile("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}"
+               : "=f"(a), "=f"(b) : "r"(v));
+}
+
+// One halving exchange of a reduce-scatter: the lanes whose `bit` is set keep the upper n words,
+// the others the lower n, and each receives its partner's copy of the words it keeps.
+template <int N>
+__device__ __forceinline__ void halve_min(uint32_t (&v)[8], int lane, int bit) {
+  const bool up = (lane & bit) != 0;
+#pragma unroll
+  for (int i = 0; i < N; ++i) {
+    const uint32_t send = up ? v[i] : v[i + N], keep = up ? v[i + N] : v[i];
+    v[i] = min_h2(keep, __shfl_xor_sync(0xffffffffu, send, bit));
+  }
+}
+
+// v[0..7] hold one f16x2 word per pass; the minimum over the LANES consecutive lanes of a group is
+// formed by halving exchanges.  Afterwards a lane holds the finished words of the passes
+//   LANES == 16: (lane & 15) >> 1 in v[0]           (both lanes of a pair hold the same one)
+//   LANES ==  8:  lane & 7        in v[0]
+//   LANES ==  4:  2 * (lane & 1) + 4 * ((lane >> 1) & 1) + j  in v[j], j = 0, 1
+template <int LANES>
+__device__ __forceinline__ void reduce_scatter_min(uint32_t (&v)[8], int lane) {
+  if (LANES == 16) {
+    halve_min<4>(v, lane, 8);
+    halve_min<2>(v, lane, 4);
+    halve_min<1>(v, lane, 2);
+    v[0] = min_h2(v[0], __shfl_xor_sync(0xffffffffu, v[0], 1));
+  } else if (LANES == 8) {
+    halve_min<4>(v, lane, 4);
+    halve_min<2>(v, lane, 2);
+    halve_min<1>(v, lane, 1);
+  } else {  // LANES == 4
+    halve_min<4>(v, lane, 2);
+    halve_min<2>(v, lane, 1);
+  }
+}
+
+// Eight codes of one row segment of fp16 weights (see the note above), packed by multiply-add.
+template <int BITS>
+__device__ __forceinline__ uint32_t pack8_h(const float (&w)[8], const float (&r)[8], const int (&nbias)[8]) {
+  constexpr int maxq = (1 << BITS) - 1;
+  uint32_t acc = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const float t = __fadd_rn(__fmaf_rn(w[k], r[k], kSnapMagic), kSnapToInt);
+    const int c = __viaddmin_s32_relu(__float_as_int(t), nbias[k], maxq);
+    acc = static_cast<uint32_t>(c) * (1u << (BITS * k)) + acc;
+  }
+  return acc;
+}
+
+template <int BITS, int G, bool DO_OC, bool DO_IC>
+__global__ void __launch_bounds__(kThreads, G == 32 ? 2 : 3)
+rtn_half_kernel(const __half* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
+                adadim_qtensor qoc, adadim_qtensor qic) {
+  constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr float rcp_maxq = 1.0f / maxq;
+  constexpr int NG = kTile / G;               // per-IC groups stacked in one tile
+  constexpr int PPG = kPasses / NG;           // passes per such group
+  constexpr int LANES = G / 8;                // lanes sharing one per-OC group
+  constexpr int HELD = LANES == 4 ? 2 : 1;    // finished per-OC groups a lane owns
+
+  __shared__ uint32_t s_mn[DO_IC ? NG : 1][8][kTile / 2];       // f16x2 column minima per warp
+  __shared__ uint32_t s_mx[DO_IC ? NG : 1][8][kTile / 2];
+  __shared__ __align__(16) float s_r[DO_IC ? NG : 1][kTile];    // reciprocal scale (0: degenerate group)
+  __shared__ __align__(16) int s_nb[DO_IC ? NG : 1][kTile];     // zero point - bits of 1.5 * 2^23
+
+  const int tid = threadIdx.x;
+  const int colvec = tid & 15, rowsub = tid >> 4;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kTile;
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * kTile;
+  const int64_t col = c0 + colvec * 8;
+  const bool col_ok = col < in;               // in % 32 == 0: a thread's 8 columns are all in or out
+  const int64_t words_per_row = in * BITS / 32;
+
+  uint4 x[kPasses];
+  uint32_t oc[8];                             // per pass: (segment minimum, -segment maximum)
+#pragma unroll
+  for (int p = 0; p < kPasses; ++p) {
+    const int64_t row = r0 + p * 16 + rowsub;
+    if (col_ok && row < out) x[p] = *reinterpret_cast<const uint4*>(W + row * ldw + col);
+    else x[p] = make_uint4(0u, 0u, 0u, 0u);   // 0 is neutral: it lies inside every [lo, hi]
+  }
+#pragma unroll
+  for (int p = 0; p < kPasses; ++p) {
+    if (DO_OC) {
+      const uint32_t mn = min_h2(min_h2(x[p].x, x[p].y), min_h2(x[p].z, x[p].w));
+      const uint32_t nmx = max_h2(max_h2(x[p].x, x[p].y), max_h2(x[p].z, x[p].w)) ^ 0x80008000u;
+      oc[p] = min_h2(__byte_perm(mn, nmx, 0x5410), __byte_perm(mn, nmx, 0x7632));
+    } else {
+      oc[p] = 0u;
+    }
+  }
+
+  // ---- per-IC statistics: column minima / maxima over each g-row group of the tile ---------
+  if (DO_IC) {
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      uint32_t cmn[4] = {x[gi * PPG].x, x[gi * PPG].y, x[gi * PPG].z, x[gi * PPG].w};
+      uint32_t cmx[4] = {cmn[0], cmn[1], cmn[2], cmn[3]};
+#pragma unroll
+      for (int pp = 1; pp < PPG; ++pp) {
+        const uint4 v = x[gi * PPG + pp];
+        cmn[0] = min_h2(cmn[0], v.x); cmn[1] = min_h2(cmn[1], v.y); cmn[2] = min_h2(cmn[2], v.z); cmn[3] = min_h2(cmn[3], v.w);
+        cmx[0] = max_h2(cmx[0], v.x); cmx[1] = max_h2(cmx[1], v.y); cmx[2] = max_h2(cmx[2], v.z); cmx[3] = max_h2(cmx[3], v.w);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        cmn[k] = min_h2(cmn[k], __shfl_xor_sync(0xffffffffu, cmn[k], 16));
+        cmx[k] = max_h2(cmx[k], __shfl_xor_sync(0xffffffffu, cmx[k], 16));
+      }
+      if (lane < 16) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          s_mn[gi][warp][colvec * 4 + k] = cmn[k];
+          s_mx[gi][warp][colvec * 4 + k] = cmx[k];
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- group parameters: each group once --------------------------------------------------------
+  float own_r[HELD];
+  int own_nb[HELD];
+#pragma unroll
+  for (int j = 0; j < HELD; ++j) { own_r[j] = 0.0f; own_nb[j] = 0; }
+  if (DO_OC) {
+    reduce_scatter_min<LANES>(oc, lane);
+#pragma unroll
+    for (int j = 0; j < HELD; ++j) {
+      const GroupParams gp = group_params(lo_h2(oc[j]), -hi_h2(oc[j]), maxq, rcp_maxq);
+      own_r[j] = gp.rcp;
+      own_nb[j] = static_cast<int>(gp.z) - kRoundMagicBits;
+      const int p = LANES == 16 ? (lane & 15) >> 1 : LANES == 8 ? (lane & 7) : 2 * (lane & 1) + 4 * ((lane >> 1) & 1) + j;
+      const int64_t row = r0 + p * 16 + rowsub;
+      const bool writer = LANES == 16 ? (lane & 1) == 0 : true;
+      if (writer && col_ok && row < out) {
+        const int64_t idx = row * (in / G) + col / G;
+        qoc.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
+        qoc.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
+      }
+    }
+  }
+  if (DO_IC) {
+    for (int t = tid; t < NG * kTile; t += kThreads) {
+      const int gi = t / kTile, c = t % kTile;
+      uint32_t mn2 = s_mn[gi][0][c >> 1], mx2 = s_mx[gi][0][c >> 1];
+#pragma unroll
+      for (int wv = 1; wv < 8; ++wv) {
+        mn2 = min_h2(mn2, s_mn[gi][wv][c >> 1]);
+        mx2 = max_h2(mx2, s_mx[gi][wv][c >> 1]);
+      }
+      const float mn = (c & 1) ? hi_h2(mn2) : lo_h2(mn2), mx = (c & 1) ? hi_h2(mx2) : lo_h2(mx2);
+      const GroupParams gp = group_params(mn, mx, maxq, rcp_maxq);
+      s_r[gi][c] = gp.rcp;
+      s_nb[gi][c] = static_cast<int>(gp.z) - kRoundMagicBits;
+      const int64_t grow = r0 / G + gi;
+      if (c0 + c < in && grow * G < out) {
+        qic.scales[grow * in + c0 + c] = __half_as_ushort(__float2half_rn(gp.s));
+        qic.zeros[grow * in + c0 + c] = __half_as_ushort(__float2half_rn(gp.z));
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- codes ------------------------------------------------------------------------------
+#pragma unroll
+  for (int gi = 0; gi < NG; ++gi) {
+    float ic_r[8];
+    int ic_nb[8];
+    if (DO_IC) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        ic_r[k] = s_r[gi][colvec * 8 + k];
+        ic_nb[k] = s_nb[gi][colvec * 8 + k];
+      }
+    }
+#pragma unroll
+    for (int pp = 0; pp < PPG; ++pp) {
+      const int p = gi * PPG + pp;
+      const int64_t row = r0 + p * 16 + rowsub;
+      const bool ok = col_ok && row < out;
+      float w[8];
+      widen_h2(x[p].x, w[0], w[1]);
+      widen_h2(x[p].y, w[2], w[3]);
+      widen_h2(x[p].z, w[4], w[5]);
+      widen_h2(x[p].w, w[6], w[7]);
+      if (DO_OC) {
+        // the lane that owns (this row, this group) of pass p, and the slot it keeps it in
+        const int base = lane & ~(LANES - 1);
+        const int src = LANES == 16 ? base | (p << 1) : LANES == 8 ? base | p : base | (((p >> 2) & 1) << 1) | ((p >> 1) & 1);
+        const int slot = LANES == 4 ? (p & 1) : 0;
+        const float rr = __shfl_sync(0xffffffffu, own_r[slot], src);
+        const int nbv = __shfl_sync(0xffffffffu, own_nb[slot], src);
+        float r8[8];
+        int nb8[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { r8[k] = rr; nb8[k] = nbv; }
+        store_codes<BITS>(pack8_h<BITS>(w, r8, nb8), qoc.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
+      }
+      if (DO_IC) {
+        store_codes<BITS>(pack8_h<BITS>(w, ic_r, ic_nb), qic.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
+      }
+    }
+  }
+}
+
+template <int BITS, int G>
+void launch_dims(const __half* W, int64_t out, int64_t in, int64_t ldw, int dim,
+                 const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  dim3 grid(static_cast<unsigned>((in + kTile - 1) / kTile), static_cast<unsigned>((out + kTile - 1) / kTile));
+  if (dim == ADADIM_DIM_BOTH)
+    rtn_half_kernel<BITS, G, true, true><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+  else if (dim == ADADIM_DIM_OC)
+    rtn_half_kernel<BITS, G, true, false><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+  else
+    rtn_half_kernel<BITS, G, false, true><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+}
+
 template <typename T, int BITS, int G>
 void launch_dims(const T* W, int64_t out, int64_t in, int64_t ldw, int dim,
                  const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
@@ -196,6 +450,14 @@ void launch_group(const T* W, int64_t out, int64_t in, int64_t ldw, int group, i
   if (group == 128) launch_dims<T, BITS, 128>(W, out, in, ldw, dim, qoc, qic, st);
   else if (group == 64) launch_dims<T, BITS, 64>(W, out, in, ldw, dim, qoc, qic, st);
   else launch_dims<T, BITS, 32>(W, out, in, ldw, dim, qoc, qic, st);
+}
+
+template <int BITS>
+void launch_group_half(const __half* W, int64_t out, int64_t in, int64_t ldw, int group, int dim,
+                       const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  if (group == 128) launch_dims<BITS, 128>(W, out, in, ldw, dim, qoc, qic, st);
+  else if (group == 64) launch_dims<BITS, 64>(W, out, in, ldw, dim, qoc, qic, st);
+  else launch_dims<BITS, 32>(W, out, in, ldw, dim, qoc, qic, st);
 }
 
 template <int BITS>
@@ -229,8 +491,8 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ codes, int64_t out, i
 int rtn_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, int bits, int group, int dim,
                const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
   if (wdtype == ADADIM_F16) {
-    if (bits == 3) launch_group<__half, 3>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
-    else launch_group<__half, 4>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
+    if (bits == 3) launch_group_half<3>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
+    else launch_group_half<4>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
   } else {
     if (bits == 3) launch_group<float, 3>(static_cast<const float*>(W), out, in, ldw, group, dim, qoc, qic, st);
     else launch_group<float, 4>(static_cast<const float*>(W), out, in, ldw, group, dim, qoc, qic, st);
