@@ -249,21 +249,26 @@ __device__ __forceinline__ void reduce_scatter_min(uint32_t (&v)[8], int lane) {
 }
 
 // Eight codes of one row segment of fp16 weights (see the note above), packed by multiply-add.
+// The two roundings run two weights at a time on the packed fp32x2 forms of fma and add; each
+// half is the IEEE operation, so nothing changes numerically.
 template <int BITS>
-__device__ __forceinline__ uint32_t pack8_h(const float (&w)[8], const float (&r)[8], const int (&nbias)[8]) {
+__device__ __forceinline__ uint32_t pack8_h(const float2 (&w)[4], const float2 (&r)[4], const int (&nbias)[8]) {
   constexpr int maxq = (1 << BITS) - 1;
+  const float2 snap = make_float2(kSnapMagic, kSnapMagic), to_int = make_float2(kSnapToInt, kSnapToInt);
   uint32_t acc = 0;
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const float t = __fadd_rn(__fmaf_rn(w[k], r[k], kSnapMagic), kSnapToInt);
-    const int c = __viaddmin_s32_relu(__float_as_int(t), nbias[k], maxq);
-    acc = static_cast<uint32_t>(c) * (1u << (BITS * k)) + acc;
+  for (int k = 0; k < 4; ++k) {
+    const float2 t = __fadd2_rn(__ffma2_rn(w[k], r[k], snap), to_int);
+    const int c0 = __viaddmin_s32_relu(__float_as_int(t.x), nbias[2 * k], maxq);
+    const int c1 = __viaddmin_s32_relu(__float_as_int(t.y), nbias[2 * k + 1], maxq);
+    acc = static_cast<uint32_t>(c0) * (1u << (BITS * 2 * k)) + acc;
+    acc = static_cast<uint32_t>(c1) * (1u << (BITS * (2 * k + 1))) + acc;
   }
   return acc;
 }
 
 template <int BITS, int G, bool DO_OC, bool DO_IC>
-__global__ void __launch_bounds__(kThreads, G == 32 ? 2 : 3)
+__global__ void __launch_bounds__(kThreads, G == 32 ? 2 : 4)
 rtn_half_kernel(const __half* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
                 adadim_qtensor qoc, adadim_qtensor qic) {
   constexpr float maxq = static_cast<float>((1 << BITS) - 1);
@@ -381,25 +386,24 @@ rtn_half_kernel(const __half* __restrict__ W, int64_t out, int64_t in, int64_t l
   // ---- codes ------------------------------------------------------------------------------
 #pragma unroll
   for (int gi = 0; gi < NG; ++gi) {
-    float ic_r[8];
+    float2 ic_r[4];
     int ic_nb[8];
     if (DO_IC) {
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        ic_r[k] = s_r[gi][colvec * 8 + k];
-        ic_nb[k] = s_nb[gi][colvec * 8 + k];
-      }
+      for (int k = 0; k < 4; ++k) ic_r[k] = make_float2(s_r[gi][colvec * 8 + 2 * k], s_r[gi][colvec * 8 + 2 * k + 1]);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) ic_nb[k] = s_nb[gi][colvec * 8 + k];
     }
 #pragma unroll
     for (int pp = 0; pp < PPG; ++pp) {
       const int p = gi * PPG + pp;
       const int64_t row = r0 + p * 16 + rowsub;
       const bool ok = col_ok && row < out;
-      float w[8];
-      widen_h2(x[p].x, w[0], w[1]);
-      widen_h2(x[p].y, w[2], w[3]);
-      widen_h2(x[p].z, w[4], w[5]);
-      widen_h2(x[p].w, w[6], w[7]);
+      float2 w[4];
+      widen_h2(x[p].x, w[0].x, w[0].y);
+      widen_h2(x[p].y, w[1].x, w[1].y);
+      widen_h2(x[p].z, w[2].x, w[2].y);
+      widen_h2(x[p].w, w[3].x, w[3].y);
       if (DO_OC) {
         // the lane that owns (this row, this group) of pass p, and the slot it keeps it in
         const int base = lane & ~(LANES - 1);
@@ -407,10 +411,12 @@ rtn_half_kernel(const __half* __restrict__ W, int64_t out, int64_t in, int64_t l
         const int slot = LANES == 4 ? (p & 1) : 0;
         const float rr = __shfl_sync(0xffffffffu, own_r[slot], src);
         const int nbv = __shfl_sync(0xffffffffu, own_nb[slot], src);
-        float r8[8];
+        float2 r8[4];
         int nb8[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { r8[k] = rr; nb8[k] = nbv; }
+        for (int k = 0; k < 4; ++k) r8[k] = make_float2(rr, rr);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) nb8[k] = nbv;
         store_codes<BITS>(pack8_h<BITS>(w, r8, nb8), qoc.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
       }
       if (DO_IC) {
