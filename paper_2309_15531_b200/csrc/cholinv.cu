@@ -198,71 +198,156 @@ build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ 
 
 // ---- factorization -------------------------------------------------------------------------
 // Diagonal block k: in-place Cholesky of the 64 x 64 block and its triangular inverse -> dinv[k].
-// Column by column (left-looking): four threads share a row's dot product; the pivot's
-// reciprocal square root scales the column.  The inverse is a forward substitution with four
-// threads per column, the column's entries spread over their registers.
-__global__ void __launch_bounds__(256)
+// The block is worked in eight sub-panels of eight columns, right-looking inside shared memory:
+//   (a) every thread factors the 8 x 8 diagonal piece redundantly in registers (the sequential
+//       chain of eight reciprocal square roots then needs no exchange between threads), and the
+//       thread that owns a row below solves its 8 entries by substitution;
+//   (b) rank-8 update of the rows and columns after the sub-panel.
+// The inverse is built in place by recursive doubling: 8 x 8 diagonal pieces by substitution
+// (one warp each, one column per lane), then three merge levels
+//   inv([[A,0],[C,B]]) = [[A^-1,0],[-B^-1 C A^-1,B^-1]].
+__global__ void __launch_bounds__(256, 2)
 potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv, int* status_dev) {
-  __shared__ double L[kNB][kNB + 1];
-  __shared__ double col[kNB];
+  constexpr int kSub = 8;
+  __shared__ double M[kNB][kNB + 1];
+  __shared__ double T[kNB / 2][kNB / 2 + 1];
   __shared__ double rdiag[kNB];          // 1 / L[j][j]
+  const int tid = threadIdx.x;
   double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
-  for (int e = threadIdx.x; e < kNB * kNB; e += 256) L[e >> 6][e & 63] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
+  for (int e = tid; e < kNB * kNB; e += 256) M[e >> 6][e & 63] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
   __syncthreads();
-  const int row = threadIdx.x >> 2, q = threadIdx.x & 3;
+
 #pragma unroll 1
-  for (int j = 0; j < kNB; ++j) {
-    double s0 = 0.0, s1 = 0.0;
-    if (row >= j) {
-      int m = q;
-      for (; m + 4 < j; m += 8) {                      // entries m = q, q+4, ... < j of the two rows
-        s0 = fma(L[row][m], L[j][m], s0);
-        s1 = fma(L[row][m + 4], L[j][m + 4], s1);
+  for (int j0 = 0; j0 < kNB; j0 += kSub) {
+    // (a) the 8 x 8 diagonal piece, in every thread
+    double d[kSub][kSub], rinv[kSub];
+#pragma unroll
+    for (int r = 0; r < kSub; ++r)
+#pragma unroll
+      for (int c = 0; c <= r; ++c) d[r][c] = M[j0 + r][j0 + c];
+    const int row = j0 + kSub + tid;                   // the row below that this thread solves
+    double x[kSub];
+    if (row < kNB) {
+#pragma unroll
+      for (int c = 0; c < kSub; ++c) x[c] = M[row][j0 + c];
+    }
+    bool bad = false;
+#pragma unroll
+    for (int c = 0; c < kSub; ++c) {
+      double piv = d[c][c];
+      if (!(piv > 0.0)) { bad = true; piv = 1.0; }
+      const double r = rsqrt(piv);
+      rinv[c] = r;
+      d[c][c] = piv * r;
+#pragma unroll
+      for (int r2 = c + 1; r2 < kSub; ++r2) d[r2][c] *= r;
+#pragma unroll
+      for (int c2 = c + 1; c2 < kSub; ++c2)
+#pragma unroll
+        for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
+    }
+    if (row < kNB) {
+#pragma unroll
+      for (int c = 0; c < kSub; ++c) {
+        double sacc = x[c];
+#pragma unroll
+        for (int m = 0; m < c; ++m) sacc = fma(-x[m], d[c][m], sacc);
+        x[c] = sacc * rinv[c];
       }
-      if (m < j) s0 = fma(L[row][m], L[j][m], s0);
     }
-    double sum = s0 + s1;
-    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-    if (q == 0 && row >= j) col[row] = L[row][j] - sum;
+    __syncthreads();                                   // every thread has read the old piece
+    if (row < kNB) {
+#pragma unroll
+      for (int c = 0; c < kSub; ++c) M[row][j0 + c] = x[c];
+    } else if (tid == 64) {
+#pragma unroll
+      for (int r = 0; r < kSub; ++r) {
+#pragma unroll
+        for (int c = 0; c <= r; ++c) M[j0 + r][j0 + c] = d[r][c];
+        rdiag[j0 + r] = rinv[r];
+      }
+      if (bad) report(status_dev, ADADIM_ERR_NOT_PD);
+    }
     __syncthreads();
-    double piv = col[j];
-    if (!(piv > 0.0)) {
-      if (threadIdx.x == 0) report(status_dev, ADADIM_ERR_NOT_PD);
-      piv = 1.0;
+    // (b) M[r][c] -= sum_m M[r][j0+m] M[c][j0+m] for lim <= c <= r; thread (ty, tx) owns rows
+    // ty + 16 i and columns tx + 16 j (neighbouring lanes read neighbouring rows: no bank conflicts)
+    const int lim = j0 + kSub;
+    if (lim < kNB) {
+      const int tx = tid & 15, ty = tid >> 4;
+      double acc[4][4] = {};
+#pragma unroll
+      for (int m = 0; m < kSub; ++m) {
+        double a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { a[i] = M[ty + 16 * i][j0 + m]; b[i] = M[tx + 16 * i][j0 + m]; }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int r = ty + 16 * i, c = tx + 16 * j;
+          if (c >= lim && c <= r) M[r][c] -= acc[i][j];
+        }
     }
-    const double r = rsqrt(piv);
-    if (q == 0 && row >= j) L[row][j] = col[row] * r;
-    if (threadIdx.x == 0) rdiag[j] = r;
     __syncthreads();
   }
-  // X = L^-1: thread (c, q) keeps X[m][c] for m = 4t + q in x[t]
+
+  // the factor goes back to the matrix (zeros above the diagonal)
+  for (int e = tid; e < kNB * kNB; e += 256) {
+    const int r = e >> 6, c = e & 63;
+    blk[static_cast<int64_t>(r) * n + c] = r >= c ? M[r][c] : 0.0;
+  }
+  __syncthreads();
+
+  // ---- inverse, in place ----------------------------------------------------------------------
   {
-    const int c = row;
-    double x[kNB / 4];
+    const int wv = tid >> 5, c = tid & 31;             // warp wv inverts piece wv, lane c its column c
+    const int o = wv * kSub;
+    double xx[kSub];
+    if (c < kSub) {
 #pragma unroll
-    for (int t = 0; t < kNB / 4; ++t) x[t] = 0.0;
-    double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
+      for (int r = 0; r < kSub; ++r) {
+        double sacc = 0.0;
 #pragma unroll
-    for (int r = 0; r < kNB; ++r) {
-      double s0 = 0.0, s1 = 0.0;
-#pragma unroll
-      for (int t = 0; t < (r + 3) / 4; ++t) {            // entries m = 4t + q < r
-        const int m = 4 * t + q;
-        const double l = m < r ? L[r][m] : 0.0;
-        if (t & 1) s1 = fma(l, x[t], s1); else s0 = fma(l, x[t], s0);
+        for (int m = 0; m < r; ++m) sacc = fma(M[o + r][o + m], xx[m], sacc);   // xx[m] == 0 for m < c
+        xx[r] = r < c ? 0.0 : ((r == c ? 1.0 : 0.0) - sacc) * rdiag[o + r];
       }
-      double sum = s0 + s1;
-      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-      const double xr = ((r == c ? 1.0 : 0.0) - sum) * rdiag[r];
-      if (q == (r & 3)) x[r >> 2] = xr;
-      if (q == 0) dk[r * kNB + c] = r < c ? 0.0 : xr;
+    }
+    __syncwarp();
+    if (c < kSub) {
+#pragma unroll
+      for (int r = 0; r < kSub; ++r) M[o + r][o + c] = xx[r];                    // zeros above the diagonal
     }
   }
-  for (int e = threadIdx.x; e < kNB * kNB; e += 256) {
-    int r = e >> 6, c = e & 63;
-    blk[static_cast<int64_t>(r) * n + c] = r >= c ? L[r][c] : 0.0;
+  __syncthreads();
+#pragma unroll 1
+  for (int sz = kSub; sz < kNB; sz *= 2) {
+    // pair p: A part rows/cols [p*2sz, p*2sz+sz), B part the next sz; T[p*sz + i][j] = (C XA)[i][j]
+    for (int e = tid; e < (kNB / 2) * sz; e += 256) {
+      const int gi = e / sz, j = e % sz, p = gi / sz, i = gi % sz;
+      const int a0 = p * 2 * sz, b0 = a0 + sz;
+      double sacc = 0.0;
+      for (int m = j; m < sz; ++m) sacc = fma(M[b0 + i][a0 + m], M[a0 + m][a0 + j], sacc);
+      T[gi][j] = sacc;
+    }
+    __syncthreads();
+    for (int e = tid; e < (kNB / 2) * sz; e += 256) {
+      const int gi = e / sz, j = e % sz, p = gi / sz, i = gi % sz;
+      const int a0 = p * 2 * sz, b0 = a0 + sz;
+      double sacc = 0.0;
+      for (int m = 0; m <= i; ++m) sacc = fma(M[b0 + i][b0 + m], T[p * sz + m][j], sacc);
+      M[b0 + i][a0 + j] = -sacc;
+    }
+    __syncthreads();
+  }
+  double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
+  for (int e = tid; e < kNB * kNB; e += 256) {
+    const int r = e >> 6, c = e & 63;
+    dk[e] = r >= c ? M[r][c] : 0.0;
   }
 }
 
@@ -305,14 +390,26 @@ group_update_kernel(double* __restrict__ A, int64_t n, int k) {
 //   A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T.
 // Row block ti meets column blocks 0 .. 2*ti+1.  The tile right of the diagonal 64-block (column
 // block 2*ti+1) only stores its lower 64 rows: the block above them must stay zero.
+// The update is issued in two parts so that the next group's factorization can start early:
+// `first_cols` launches a (kLook, row blocks) grid over the first kLook column blocks (the next
+// group's own columns); the other launch walks the whole triangle and skips those.
+constexpr int kLook = kGroup * kNB / kTN;
 __global__ void __launch_bounds__(256, 2)
-rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
+rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw, bool first_cols) {
   __shared__ TileSmem sm;
-  const int t = blockIdx.x;
-  int ti = static_cast<int>((sqrt(4.0 * t + 1.0) - 1.0) * 0.5);
-  while (ti * (ti + 1) > t) --ti;
-  while ((ti + 1) * (ti + 2) <= t) ++ti;
-  const int cj = t - ti * (ti + 1);
+  int ti, cj;
+  if (first_cols) {
+    ti = blockIdx.y;
+    cj = blockIdx.x;
+    if (cj > 2 * ti + 1) return;
+  } else {
+    const int t = blockIdx.x;
+    ti = static_cast<int>((sqrt(4.0 * t + 1.0) - 1.0) * 0.5);
+    while (ti * (ti + 1) > t) --ti;
+    while ((ti + 1) * (ti + 2) <= t) ++ti;
+    cj = t - ti * (ti + 1);
+    if (cj < kLook) return;
+  }
   const int64_t ri = e + static_cast<int64_t>(ti) * kT, rj = e + static_cast<int64_t>(cj) * kTN;
   if (rj >= n) return;
   const int vr = static_cast<int>(mn64(kT, n - ri));
@@ -452,23 +549,64 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
   const int nb = static_cast<int>(n / kNB);
   const unsigned eb = static_cast<unsigned>((n * n + 255) / 256);
 
+  // The factorization's chain of small kernels (diagonal blocks, panels, in-group updates and the
+  // rank update of the next group's own columns) runs on a high-priority stream; the rest of each
+  // group's rank update runs beside it on a second stream.  Every kernel of the chain fits on an
+  // SM next to one CTA of the rank update, so the chain is scheduled as soon as any CTA retires.
+  cudaStream_t chain = nullptr, side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_panels = nullptr, ev_rest = nullptr, ev_join = nullptr;
+  int prio_least = 0, prio_greatest = 0;
+  ADADIM_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&chain, cudaStreamNonBlocking, prio_greatest));
+  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, prio_least));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_panels, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_rest, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
+  bool rest_pending = false;
+
   damp_kernel<<<1, 256, 0, st>>>(H, n, static_cast<double>(percdamp), stats);
   build_kernel<<<eb, 256, 0, st>>>(H, n, stats, A);
+  ADADIM_CUDA_TRY(cudaEventRecord(ev_fork, st));
+  ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_fork, 0));
   for (int g0 = 0; g0 < nb; g0 += kGroup) {
     const int g1 = g0 + kGroup < nb ? g0 + kGroup : nb;
     for (int k = g0; k < g1; ++k) {
-      potrf_kernel<<<1, 256, 0, st>>>(A, n, k, dinv, status_dev);
+      potrf_kernel<<<1, 256, 0, chain>>>(A, n, k, dinv, status_dev);
       const int below = nb - k - 1;
-      if (below > 0) panel_kernel<<<below, 256, 0, st>>>(A, n, k, dinv);
+      if (below > 0) panel_kernel<<<below, 256, 0, chain>>>(A, n, k, dinv);
       const int inner = g1 - k - 1;
-      if (below > 0 && inner > 0) group_update_kernel<<<dim3(below, inner), 256, 0, st>>>(A, n, k);
+      if (below > 0 && inner > 0) group_update_kernel<<<dim3(below, inner), 256, 0, chain>>>(A, n, k);
     }
     const int64_t e = static_cast<int64_t>(g1) * kNB;
     if (e < n) {
       const int nt = static_cast<int>((n - e + kT - 1) / kT);
-      rank_update_kernel<<<nt * (nt + 1), 256, 0, st>>>(A, n, e, static_cast<int64_t>(g0) * kNB, (g1 - g0) * kNB);
+      const int64_t j0 = static_cast<int64_t>(g0) * kNB;
+      const int kw = (g1 - g0) * kNB;
+      const bool has_rest = e + kLook * kTN < n;
+      if (has_rest) ADADIM_CUDA_TRY(cudaEventRecord(ev_panels, chain));
+      // the columns updated next were last written by the previous group's side-stream launch
+      if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
+      rank_update_kernel<<<dim3(kLook, nt), 256, 0, chain>>>(A, n, e, j0, kw, true);
+      rest_pending = false;
+      if (has_rest) {
+        ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_panels, 0));
+        rank_update_kernel<<<nt * (nt + 1), 256, 0, side>>>(A, n, e, j0, kw, false);
+        ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
+        rest_pending = true;
+      }
     }
   }
+  if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
+  ADADIM_CUDA_TRY(cudaEventRecord(ev_join, chain));
+  ADADIM_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+  // destruction is deferred by the runtime until the work already enqueued has finished
+  cudaEventDestroy(ev_fork);
+  cudaEventDestroy(ev_panels);
+  cudaEventDestroy(ev_rest);
+  cudaEventDestroy(ev_join);
+  cudaStreamDestroy(chain);
+  cudaStreamDestroy(side);
   seed_kernel<<<nb, 256, 0, st>>>(A, n, dinv);
   if (n > kNB) {
     const unsigned pairs = static_cast<unsigned>((n + 2 * kNB - 1) / (2 * kNB));
