@@ -95,7 +95,7 @@ def launches_per_step(out: int, inp: int) -> int:
         for k in range(g0, g1):
             below, inner = nb - k - 1, g1 - k - 1
             factor += 1 + (1 if below > 0 else 0) + (1 if below > 0 and inner > 0 else 0)
-        factor += 1 if g1 * 64 < inp else 0              # rank-256 update
+        factor += (1 if g1 * 64 < inp else 0) + (1 if g1 * 64 + 256 < inp else 0)   # rank-256 update: next group's columns, rest
     factor += 1 + (2 if inp > 64 else 0)                 # seed, 64-level merges
     s = 128
     while s < inp:
@@ -103,7 +103,7 @@ def launches_per_step(out: int, inp: int) -> int:
         s *= 2
     factor += 1                                          # emit
     blocks = inp // 128
-    gptq = 1 + 1 + blocks + (blocks - 1) + 1           # init, U slicing, block kernels, trailing kernels, loss
+    gptq = 1 + 1 + blocks + (blocks - 1) + max(blocks - 2, 0) + 1   # init, U slicing, block kernels, next-block and rest trailing kernels, loss
     hessian = 2 if inp > 256 else 1
     rtn = 1
     score = 1 + 1 + 1                                  # difference kernel, Gram product, finalize

@@ -219,47 +219,49 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
 
 #pragma unroll 1
   for (int j0 = 0; j0 < kNB; j0 += kSub) {
-    // (a) the 8 x 8 diagonal piece, in every thread
+    // (a) the 8 x 8 diagonal piece, in every thread of the two warps that own the rows below
     double d[kSub][kSub], rinv[kSub];
-#pragma unroll
-    for (int r = 0; r < kSub; ++r)
-#pragma unroll
-      for (int c = 0; c <= r; ++c) d[r][c] = M[j0 + r][j0 + c];
     const int row = j0 + kSub + tid;                   // the row below that this thread solves
     double x[kSub];
-    if (row < kNB) {
-#pragma unroll
-      for (int c = 0; c < kSub; ++c) x[c] = M[row][j0 + c];
-    }
     bool bad = false;
+    if (tid < 64) {
 #pragma unroll
-    for (int c = 0; c < kSub; ++c) {
-      double piv = d[c][c];
-      if (!(piv > 0.0)) { bad = true; piv = 1.0; }
-      const double r = rsqrt(piv);
-      rinv[c] = r;
-      d[c][c] = piv * r;
+      for (int r = 0; r < kSub; ++r)
 #pragma unroll
-      for (int r2 = c + 1; r2 < kSub; ++r2) d[r2][c] *= r;
+        for (int c = 0; c <= r; ++c) d[r][c] = M[j0 + r][j0 + c];
+      if (row < kNB) {
 #pragma unroll
-      for (int c2 = c + 1; c2 < kSub; ++c2)
-#pragma unroll
-        for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
-    }
-    if (row < kNB) {
+        for (int c = 0; c < kSub; ++c) x[c] = M[row][j0 + c];
+      }
 #pragma unroll
       for (int c = 0; c < kSub; ++c) {
-        double sacc = x[c];
+        double piv = d[c][c];
+        if (!(piv > 0.0)) { bad = true; piv = 1.0; }
+        const double r = rsqrt(piv);
+        rinv[c] = r;
+        d[c][c] = piv * r;
 #pragma unroll
-        for (int m = 0; m < c; ++m) sacc = fma(-x[m], d[c][m], sacc);
-        x[c] = sacc * rinv[c];
+        for (int r2 = c + 1; r2 < kSub; ++r2) d[r2][c] *= r;
+#pragma unroll
+        for (int c2 = c + 1; c2 < kSub; ++c2)
+#pragma unroll
+          for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
+      }
+      if (row < kNB) {
+#pragma unroll
+        for (int c = 0; c < kSub; ++c) {
+          double sacc = x[c];
+#pragma unroll
+          for (int m = 0; m < c; ++m) sacc = fma(-x[m], d[c][m], sacc);
+          x[c] = sacc * rinv[c];
+        }
       }
     }
     __syncthreads();                                   // every thread has read the old piece
     if (row < kNB) {
 #pragma unroll
       for (int c = 0; c < kSub; ++c) M[row][j0 + c] = x[c];
-    } else if (tid == 64) {
+    } else if (tid == 63) {                            // never owns a row: j0 + 8 + 63 > 63
 #pragma unroll
       for (int r = 0; r < kSub; ++r) {
 #pragma unroll
@@ -296,9 +298,12 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
     __syncthreads();
   }
 
-  // the factor goes back to the matrix (zeros above the diagonal)
+  // the factor goes back to the matrix; above the diagonal it is zero there and, from here on, in
+  // M too (the updates that produced this block left symmetric leftovers there, and the merges
+  // below sum over whole rows and columns)
   for (int e = tid; e < kNB * kNB; e += 256) {
     const int r = e >> 6, c = e & 63;
+    if (r < c) M[r][c] = 0.0;
     blk[static_cast<int64_t>(r) * n + c] = r >= c ? M[r][c] : 0.0;
   }
   __syncthreads();
@@ -326,21 +331,45 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
   __syncthreads();
 #pragma unroll 1
   for (int sz = kSub; sz < kNB; sz *= 2) {
-    // pair p: A part rows/cols [p*2sz, p*2sz+sz), B part the next sz; T[p*sz + i][j] = (C XA)[i][j]
-    for (int e = tid; e < (kNB / 2) * sz; e += 256) {
-      const int gi = e / sz, j = e % sz, p = gi / sz, i = gi % sz;
-      const int a0 = p * 2 * sz, b0 = a0 + sz;
-      double sacc = 0.0;
-      for (int m = j; m < sz; ++m) sacc = fma(M[b0 + i][a0 + m], M[a0 + m][a0 + j], sacc);
-      T[gi][j] = sacc;
+    // pair p: A part rows/cols [p*2sz, p*2sz+sz), B part the next sz; T[p*sz + i][j] = (C XA)[i][j].
+    // A thread works on up to four elements at once (32*sz/256 = sz/8 <= 4) so that the dependent
+    // chains of multiply-adds overlap; terms outside the triangles are zeros in M.
+    const int per = sz / 8;                            // elements per thread: 1, 2, 4
+    {
+      int gi[4], jj[4];
+      double sacc[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int e = tid + 256 * (u < per ? u : 0); gi[u] = e / sz; jj[u] = e % sz; }
+      for (int m = 0; m < sz; ++m) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int p = gi[u] / sz, i = gi[u] % sz, a0 = p * 2 * sz, b0 = a0 + sz;
+          sacc[u] = fma(M[b0 + i][a0 + m], M[a0 + m][a0 + jj[u]], sacc[u]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) if (u < per) T[gi[u]][jj[u]] = sacc[u];
     }
     __syncthreads();
-    for (int e = tid; e < (kNB / 2) * sz; e += 256) {
-      const int gi = e / sz, j = e % sz, p = gi / sz, i = gi % sz;
-      const int a0 = p * 2 * sz, b0 = a0 + sz;
-      double sacc = 0.0;
-      for (int m = 0; m <= i; ++m) sacc = fma(M[b0 + i][b0 + m], T[p * sz + m][j], sacc);
-      M[b0 + i][a0 + j] = -sacc;
+    {
+      int gi[4], jj[4];
+      double sacc[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int e = tid + 256 * (u < per ? u : 0); gi[u] = e / sz; jj[u] = e % sz; }
+      for (int m = 0; m < sz; ++m) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int p = gi[u] / sz, i = gi[u] % sz, b0 = p * 2 * sz + sz;
+          sacc[u] = fma(M[b0 + i][b0 + m], T[p * sz + m][jj[u]], sacc[u]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (u < per) {
+          const int p = gi[u] / sz, i = gi[u] % sz, a0 = p * 2 * sz, b0 = a0 + sz;
+          M[b0 + i][a0 + jj[u]] = -sacc[u];
+        }
+      }
     }
     __syncthreads();
   }
@@ -472,9 +501,11 @@ merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T
 __global__ void __launch_bounds__(256, 2)
 merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T) {      // s >= 128
   __shared__ TileSmem sm;
-  const int ctiles = static_cast<int>(s / kTN);
   const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  const int r = blockIdx.x / ctiles, c = blockIdx.x % ctiles;          // 128-row block, 64-column block
+  // 128-row block r, 64-column block c; the reduction length s - 64 c falls with c, so tiles are
+  // handed out column block by column block: the longest ones start first
+  const int rtiles = static_cast<int>(s / kT);
+  const int r = blockIdx.x % rtiles, c = blockIdx.x / rtiles;
   const int64_t sB = mn64(s, n - b0);
   if (static_cast<int64_t>(r) * kT >= sB) return;
   const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
@@ -495,7 +526,9 @@ merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __rest
   __shared__ TileSmem sm;
   const int ctiles = static_cast<int>(s / kTN);
   const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  const int r = blockIdx.x / ctiles, c = blockIdx.x % ctiles;
+  // the reduction length 128 (r + 1) grows with the row block: the last row blocks start first
+  const int rtiles = static_cast<int>(s / kT);
+  const int r = rtiles - 1 - static_cast<int>(blockIdx.x) / ctiles, c = blockIdx.x % ctiles;
   const int64_t sB = mn64(s, n - b0);
   if (static_cast<int64_t>(r) * kT >= sB) return;
   const int64_t row0 = b0 + static_cast<int64_t>(r) * kT;

@@ -25,7 +25,7 @@ struct TrailPlan {
 int trail_split_u(const float* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st);
 int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
                const __nv_bfloat16* const u[3]);
-int trail_launch(const TrailPlan& plan, int i1, int* status_dev, cudaStream_t st);
+int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_ctas, int* status_dev, cudaStream_t st);
 
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
@@ -66,6 +66,12 @@ struct BlockArgs {
   int64_t out, in;
   int i1;                    // first column of the block
 };
+
+__device__ __forceinline__ int ordered_key(float v) {
+  const int b = __float_as_int(v);
+  return b ^ ((b >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float from_ordered_key(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7fffffff)); }
 
 template <int BITS, int G>
 __global__ void __launch_bounds__(kBlk, 1)
@@ -133,12 +139,11 @@ block_kernel(const BlockArgs a) {
           q.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
         }
       } else {                                       // per-IC: parameters of this column's g-row groups
-        float mn = w[ii], mx = w[ii];
-#pragma unroll
-        for (int m = 16; m > 0; m >>= 1) {
-          mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, m));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
-        }
+        // warp minimum and maximum in one reduction instruction each, on a key that orders
+        // floats as signed integers (negative values have their magnitude bits flipped)
+        const int key = ordered_key(w[ii]);
+        float mn = from_ordered_key(__reduce_min_sync(0xffffffffu, key));
+        float mx = from_ordered_key(__reduce_max_sync(0xffffffffu, key));
         if (G > 32) {
           float* slot = red + (ii & 1) * 8;
           if (lane == 0) { slot[warp * 2] = mn; slot[warp * 2 + 1] = mx; }
@@ -264,7 +269,7 @@ GptqLayout gptq_layout(int64_t out, int64_t in) {
   GptqLayout L;
   size_t off = 0;
   L.wc_off = off;     off += round_up(static_cast<size_t>(2) * out * in * 4, 256);
-  L.err_piece = round_up(static_cast<size_t>(2) * out * kBlk * 2, 1024);
+  L.err_piece = round_up(static_cast<size_t>(2) * 2 * out * kBlk * 2, 1024);      // two alternating sets
   L.err_off = off;    off += 3 * L.err_piece;
   L.up_piece = round_up(static_cast<size_t>(in) * in * 2, 1024);
   L.up_off = off;     off += 3 * L.up_piece;
@@ -321,22 +326,68 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   TrailPlan plan;
   rc0 = trail_plan(&plan, a.Wc, static_cast<int64_t>(ndim) * out, in, ep, up);
   if (rc0 != ADADIM_OK) return rc0;
+  // Block b+1 only needs its own 128 columns from block b's trailing update.  That part runs on a
+  // high-priority stream together with the block kernels; the rest of each trailing update runs
+  // beside the next block kernel on a second stream, on few enough CTAs to leave it room.  The
+  // error pieces alternate between two sets, so a block kernel never overwrites what the other
+  // stream still reads.
+  cudaStream_t chain = nullptr, side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_block = nullptr, ev_rest = nullptr, ev_join = nullptr;
+  int prio_least = 0, prio_greatest = 0;
+  ADADIM_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&chain, cudaStreamNonBlocking, prio_greatest));
+  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, prio_least));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_block, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_rest, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
+  ADADIM_CUDA_TRY(cudaEventRecord(ev_fork, st));
+  ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_fork, 0));
+  const int64_t rows_total = static_cast<int64_t>(ndim) * out;
+  const int block_ctas = slabs * ndim;
+  const int rest_ctas = plan.sm_count - block_ctas > 0 ? plan.sm_count - block_ctas : 1;
+  __nv_bfloat16* ep_base[3] = {a.Ep[0], a.Ep[1], a.Ep[2]};
+  bool rest_pending = false;
   for (int i1 = 0; i1 < in; i1 += kBlk) {
     a.i1 = i1;
+    for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows_total * kBlk;
     int rc;
     if (bits == 3) {
-      rc = group == 128 ? block_launch<3, 128>(a, slabs, ndim, st) : group == 64 ? block_launch<3, 64>(a, slabs, ndim, st)
-                                                                                 : block_launch<3, 32>(a, slabs, ndim, st);
+      rc = group == 128 ? block_launch<3, 128>(a, slabs, ndim, chain) : group == 64 ? block_launch<3, 64>(a, slabs, ndim, chain)
+                                                                                    : block_launch<3, 32>(a, slabs, ndim, chain);
     } else {
-      rc = group == 128 ? block_launch<4, 128>(a, slabs, ndim, st) : group == 64 ? block_launch<4, 64>(a, slabs, ndim, st)
-                                                                                 : block_launch<4, 32>(a, slabs, ndim, st);
+      rc = group == 128 ? block_launch<4, 128>(a, slabs, ndim, chain) : group == 64 ? block_launch<4, 64>(a, slabs, ndim, chain)
+                                                                                    : block_launch<4, 32>(a, slabs, ndim, chain);
     }
     if (rc != ADADIM_OK) return rc;
-    if (in - i1 - kBlk > 0) {
-      rc = trail_launch(plan, i1, status_dev, st);
+    const int tiles_after = static_cast<int>((in - i1 - kBlk) / kBlk);
+    if (tiles_after > 0) {
+      if (tiles_after > 1) ADADIM_CUDA_TRY(cudaEventRecord(ev_block, chain));
+      // the next block's columns were last written by the previous block's side-stream launch
+      if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
+      rest_pending = false;
+      rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, plan.sm_count, status_dev, chain);
       if (rc != ADADIM_OK) return rc;
+      if (tiles_after > 1) {
+        ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_block, 0));
+        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1, rest_ctas, status_dev, side);
+        if (rc != ADADIM_OK) return rc;
+        ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
+        rest_pending = true;
+      }
     }
   }
+  if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
+  ADADIM_CUDA_TRY(cudaEventRecord(ev_join, chain));
+  ADADIM_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+  // destruction is deferred by the runtime until the work already enqueued has finished
+  cudaEventDestroy(ev_fork);
+  cudaEventDestroy(ev_block);
+  cudaEventDestroy(ev_rest);
+  cudaEventDestroy(ev_join);
+  cudaStreamDestroy(chain);
+  cudaStreamDestroy(side);
+  for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k];
   if (gptq_loss != nullptr) loss_kernel<<<1, 32, 0, st>>>(a.loss_part, ndim, slabs, a, gptq_loss);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }

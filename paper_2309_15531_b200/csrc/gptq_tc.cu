@@ -38,6 +38,7 @@ struct TrailParams {
   int64_t c0;           // first column to update
   int i1;               // first row of U's block
   int ntiles;           // 128-column tiles from c0
+  int e_row0;           // first row of this block's error pieces (the pieces are kept in two alternating sets)
   int* status_dev;
 };
 
@@ -91,7 +92,7 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
       ptx::mbar_arrive_expect_tx(a_full, kABytes);
       for (int pc = 0; pc < 3; ++pc)
         for (int kh = 0; kh < 2; ++kh)
-          ptx::tma_load_2d(a_smem + (pc * 2 + kh) * kAPiece, tmE[pc], kh * 64, mrow, a_full);
+          ptx::tma_load_2d(a_smem + (pc * 2 + kh) * kAPiece, tmE[pc], kh * 64, p.e_row0 + mrow, a_full);
       int stage = 0;
       uint32_t phase = 0;
       int last_phase[kBStages];
@@ -278,7 +279,7 @@ int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const
   plan->rows_total = rows_total;
   plan->in = in;
   for (int k = 0; k < 3; ++k) {
-    int rc = make_tmap_bf16(&plan->e[k], e[k], 128, static_cast<uint64_t>(rows_total), 256, 128);
+    int rc = make_tmap_bf16(&plan->e[k], e[k], 128, static_cast<uint64_t>(2 * rows_total), 256, 128);   // two sets
     if (rc != ADADIM_OK) return rc;
     rc = make_tmap_bf16(&plan->u[k], u[k], static_cast<uint64_t>(in), static_cast<uint64_t>(in),
                         static_cast<uint64_t>(in) * 2, 32);
@@ -292,17 +293,20 @@ int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const
   return ADADIM_OK;
 }
 
-int trail_launch(const TrailPlan& plan, int i1, int* status_dev, cudaStream_t st) {
+// Updates `ntiles` 128-column tiles starting at column c0 with the errors of the block whose first
+// column is i1 (error set i1/128 & 1), on at most max_ctas CTAs.
+int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_ctas, int* status_dev, cudaStream_t st) {
   TrailParams p;
   p.Wc = plan.Wc;
   p.in = plan.in;
-  p.c0 = static_cast<int64_t>(i1) + 128;
+  p.c0 = c0;
   p.i1 = i1;
-  p.ntiles = static_cast<int>((plan.in - p.c0 + kTileN - 1) / kTileN);
+  p.ntiles = ntiles;
+  p.e_row0 = static_cast<int>(((i1 / 128) & 1) * plan.rows_total);
   p.status_dev = status_dev;
   if (p.ntiles <= 0) return ADADIM_OK;
   const int mblocks = static_cast<int>(plan.rows_total / 128);
-  int nsplit = plan.sm_count / mblocks;
+  int nsplit = max_ctas / mblocks;
   if (nsplit < 1) nsplit = 1;
   if (nsplit > p.ntiles) nsplit = p.ntiles;
   trail_kernel<<<dim3(nsplit, mblocks), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],

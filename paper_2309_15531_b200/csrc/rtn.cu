@@ -192,7 +192,6 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
 //    fma(w, rcp, 192) rounds p to a multiple of 2^-16: an exact tie comes out as exactly m + 1/2,
 //    everything else stays on its side of every m + 1/2.  Adding 1.5 * 2^23 - 192 then rounds
 //    that to an integer, ties to even, which is rint of the correctly rounded quotient.
-constexpr int kPrefetchDistance = 600;                   // a little more than the CTAs resident on 148 SMs
 constexpr float kSnapMagic = 192.0f;                     // 1.5 * 2^7: ulp 2^-16 in [128, 256)
 constexpr float kSnapToInt = 12582912.0f - 192.0f;       // exact in binary32
 
@@ -300,19 +299,6 @@ rtn_half_kernel(const __half* __restrict__ W, int64_t out, int64_t in, int64_t l
     const int64_t row = r0 + p * 16 + rowsub;
     if (col_ok && row < out) x[p] = *reinterpret_cast<const uint4*>(W + row * ldw + col);
     else x[p] = make_uint4(0u, 0u, 0u, 0u);   // 0 is neutral: it lies inside every [lo, hi]
-  }
-  // Ask L2 for the tile that a CTA launched about one residency later will read (CTAs start in
-  // grid order), so that its loads find the lines on chip.  One request per 128-byte line.
-  {
-    const int64_t ahead = static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x + kPrefetchDistance;
-    const int64_t pr0 = ahead / gridDim.x * kTile, pc = ahead % gridDim.x * kTile + colvec * 8;
-    if ((colvec & 7) == 0 && pc < in) {
-#pragma unroll
-      for (int p = 0; p < kPasses; ++p) {
-        const int64_t row = pr0 + p * 16 + rowsub;
-        if (row < out) asm volatile("prefetch.global.L2 [%0];" ::"l"(W + row * ldw + pc));
-      }
-    }
   }
 #pragma unroll
   for (int p = 0; p < kPasses; ++p) {

@@ -77,4 +77,4 @@ def test_launch_count_matches_the_host_logic():
     # panels remain in the group, one rank-256 update per finished group with columns to its right
     assert bench.launches_per_step(4096, 128) > 0
     n = bench.launches_per_step(4096, 4096)
-    assert n == 281                                    # Hessian 2, RTN 1, scorer 3 + 3, factor 206, GPTQ 66
+    assert n == 325                                    # Hessian 2, RTN 1, scorer 3 + 3, factor 220, GPTQ 96
