@@ -275,6 +275,73 @@ def quantize_gptq(W, H, bits, group, dim, percdamp=0.01, U=None, dead=None):
             "Q": Q, "Err": Err, "loss": 0.5 * float(np.sum(Err * Err))}
 
 
+def activation_order(H):
+    """Column order of activation reordering (Section 2.2; Appendix A.1): input channels by
+    descending activation magnitude, i.e. descending diag(H) after the dead-column fix, equal
+    values keeping their original order."""
+    d = np.diag(np.asarray(H, dtype=np.float64)).copy()
+    d[d == 0.0] = 1.0
+    return np.argsort(-d, kind="stable")
+
+
+def quantize_gptq_reordered(W, H, bits, group, dim, percdamp=0.01, static_groups=False):
+    """GPTQ with activation reordering (Section 2.2, Appendix A.1).
+
+    The columns of W (and rows/columns of H) are taken in the order of activation_order(H):
+    the method is the plain one applied to W[:, perm] and H[perm][:, perm]; codes, the
+    dequantized weights and the per-column errors are returned at the columns' original
+    positions.
+
+    dim == "ic": group statistics are dynamic as before (the g rows of the column being
+    quantized, from the current weights); a column's scale and zero are stored at its original
+    position, so the parameter layout [out/g, in] is unchanged.
+    dim == "oc": only with static_groups=True (the hardware-efficient variant of Section 2.2):
+    the parameters of every group of g consecutive original columns are fixed before anything
+    is reordered or updated, from the original weights, and a column uses the parameters of
+    the group it originally belongs to.
+    Returns the same dict as quantize_gptq plus "perm".
+    """
+    Wf = np.asarray(W).astype(F32)
+    out, inp = Wf.shape
+    Hd, dead = damped_hessian(H, percdamp)
+    perm = activation_order(H)
+    Hp = Hd[np.ix_(perm, perm)]
+    U = cholesky_inverse_factor(Hp)
+    Wc = np.array(Wf[:, perm], dtype=np.float64)
+    Wc[:, dead[perm]] = 0.0
+    codes = np.zeros((out, inp), dtype=np.uint8)
+    Q = np.zeros((out, inp), dtype=F32)
+    Err = np.zeros((out, inp), dtype=np.float64)
+    if dim == "oc":
+        if not static_groups:
+            raise ValueError("per-OC reordering is defined here only with static groups")
+        assert inp % group == 0
+        G0 = Wf.reshape(out, inp // group, group)
+        S, Z, B = group_params(G0.min(axis=2), G0.max(axis=2), bits)
+    else:
+        assert out % group == 0
+        S = np.zeros((out // group, inp), dtype=F32)
+        Z = np.zeros((out // group, inp), dtype=F32)
+    for i in range(inp):
+        c0 = int(perm[i])                       # original position of the column quantized now
+        w32 = Wc[:, i].astype(F32)
+        if dim == "oc":
+            se, ze, be = S[:, c0 // group], Z[:, c0 // group], B[:, c0 // group]
+        else:
+            col = w32.reshape(out // group, group)
+            s, z, bad = group_params(col.min(axis=1), col.max(axis=1), bits)
+            S[:, c0], Z[:, c0] = s, z
+            se, ze, be = np.repeat(s, group), np.repeat(z, group), np.repeat(bad, group)
+        c = encode(w32, se, ze, bits, be)
+        q = dequant(c, se, ze)
+        codes[:, c0], Q[:, c0] = c, q
+        e = (Wc[:, i] - q.astype(np.float64)) / U[i, i]
+        Err[:, c0] = e
+        Wc[:, i:] -= np.outer(e, U[i, i:])
+    return {"codes": codes, "scales": S.astype(np.float16), "zeros": Z.astype(np.float16),
+            "Q": Q, "Err": Err, "loss": 0.5 * float(np.sum(Err * Err)), "perm": perm}
+
+
 # ---------------------------------------------------------------------------
 # Flows (Section 3.3, Appendix B).
 # ---------------------------------------------------------------------------

@@ -222,3 +222,98 @@ def test_flows():
     b2, e2, r2 = O.gptq_both(W, H, 3, 128)
     assert b2 == O.select_dim(e2["oc"], e2["ic"])
     assert np.array_equal(r2["ic"]["codes"], O.quantize_gptq(W, H, 3, 128, "ic")["codes"])
+
+
+# ----------------------------------------------------------------------------- activation reordering
+
+def test_activation_order_is_descending_and_stable():
+    H = np.diag([3.0, 9.0, 0.0, 9.0, 0.5, 1.0])
+    # the dead column counts as 1 (its diagonal is set to 1 before anything else), ties keep their order
+    assert list(O.activation_order(H)) == [1, 3, 0, 2, 5, 4]
+    _, X = _layer(8, 64, 300, outliers=(3, 17), scale=40.0)
+    perm = O.activation_order(O.hessian(X))
+    assert set(perm[:2]) == {3, 17}                   # the salient channels are quantized first
+    assert sorted(perm) == list(range(64))
+
+
+@pytest.mark.parametrize("dim", ["oc", "ic"])
+def test_uncorrelated_channels_reduce_to_rtn_in_any_order(dim):
+    """With a diagonal Hessian nothing propagates (U is diagonal), so every column is rounded as it
+    stands whatever the order: the result must be RTN's, at the original positions."""
+    W = (RNG.standard_normal((64, 96)) * 0.02).astype(np.float32)
+    H = np.diag(RNG.uniform(0.5, 50.0, 96))
+    r = O.quantize_gptq_reordered(W, H, 3, 32, dim, static_groups=(dim == "oc"))
+    assert not np.array_equal(r["perm"], np.arange(96))
+    t = O.quantize_rtn(W, 3, 32, dim)
+    for k in ("codes", "scales", "zeros", "Q"):
+        assert np.array_equal(r[k], t[k]), k
+
+
+def test_reordered_ic_is_the_plain_method_on_the_permuted_problem():
+    W, X = _layer(64, 96, 300, outliers=(5, 40), scale=25.0)
+    H = O.hessian(X)
+    r = O.quantize_gptq_reordered(W, H, 3, 32, "ic")
+    perm = r["perm"]
+    p = O.quantize_gptq(np.ascontiguousarray(W[:, perm]), H[np.ix_(perm, perm)], 3, 32, "ic")
+    assert np.array_equal(r["codes"][:, perm], p["codes"])
+    assert np.array_equal(r["scales"][:, perm].view(np.uint16), p["scales"].view(np.uint16))
+    assert np.array_equal(r["zeros"][:, perm].view(np.uint16), p["zeros"].view(np.uint16))
+    assert np.array_equal(r["Q"][:, perm], p["Q"])
+    assert r["loss"] == pytest.approx(p["loss"], rel=1e-12)
+    # and reordering changes the outcome (otherwise the test above proves nothing)
+    assert not np.array_equal(r["codes"], O.quantize_gptq(W, H, 3, 32, "ic")["codes"])
+
+
+def _elimination_in_order(W, Hd, bits, group, dim, order, static=None):
+    """Greedy coordinate elimination in the ORIGINAL index space: coordinates are fixed in the
+    given order, the inverse Hessian of the coordinates still free is kept explicitly (rows and
+    columns of fixed ones become zero through the downdate), no array is ever permuted."""
+    Wc = W.astype(np.float64).copy()
+    out, inp = Wc.shape
+    Hinv = np.linalg.inv(Hd)
+    codes = np.zeros((out, inp), np.uint8)
+    for c0 in order:
+        w32 = Wc[:, c0].astype(np.float32)
+        if dim == "oc":
+            s, z, bad = (a[:, c0 // group] for a in static)
+        else:
+            col = w32.reshape(out // group, group)
+            s, z, bad = (np.repeat(a, group) for a in O.group_params(col.min(1), col.max(1), bits))
+        c = O.encode(w32, s, z, bits, bad)
+        codes[:, c0] = c
+        q = O.dequant(c, s, z).astype(np.float64)
+        d = Hinv[c0, c0]
+        Wc -= np.outer((Wc[:, c0] - q) / d, Hinv[c0, :])
+        Hinv = Hinv - np.outer(Hinv[:, c0], Hinv[c0, :]) / d
+    return codes
+
+
+@pytest.mark.parametrize("dim", ["oc", "ic"])
+def test_reordered_matches_elimination_in_original_coordinates(dim):
+    W, X = _layer(32, 48, 200, outliers=(3, 30), scale=20.0)
+    H = O.hessian(X)
+    Hd, _ = O.damped_hessian(H, 0.01)
+    order = O.activation_order(H)
+    static = None
+    if dim == "oc":
+        G0 = W.reshape(32, 3, 16)
+        static = O.group_params(G0.min(2), G0.max(2), 3)
+    r = O.quantize_gptq_reordered(W, H, 3, 16, dim, static_groups=(dim == "oc"))
+    assert np.array_equal(r["codes"], _elimination_in_order(W, Hd, 3, 16, dim, order, static))
+
+
+@pytest.mark.parametrize("dim", ["oc", "ic"])
+def test_reordered_loss_identity_and_static_parameters(dim):
+    W, X = _layer(64, 96, 300, outliers=(5, 40), scale=25.0)
+    H = O.hessian(X)
+    Hd, _ = O.damped_hessian(H, 0.01)
+    r = O.quantize_gptq_reordered(W, H, 3, 32, dim, static_groups=(dim == "oc"))
+    D = W.astype(np.float64) - r["Q"].astype(np.float64)
+    assert r["loss"] == pytest.approx(0.5 * float(np.sum((D @ Hd) * D)), rel=1e-9)
+    assert np.array_equal(O.dequantize(r["codes"], r["scales"], r["zeros"], 32, dim), r["Q"])
+    if dim == "oc":                                   # static groups: the parameters are RTN's
+        t = O.quantize_rtn(W, 3, 32, "oc")
+        assert np.array_equal(r["scales"].view(np.uint16), t["scales"].view(np.uint16))
+        assert np.array_equal(r["zeros"].view(np.uint16), t["zeros"].view(np.uint16))
+    with pytest.raises(ValueError):
+        O.quantize_gptq_reordered(W, H, 3, 32, "oc", static_groups=False)
