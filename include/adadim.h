@@ -144,6 +144,31 @@ ADADIM_API int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int6
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * GPTQ with activation reordering (Section 2.2; Appendix A.1): the input channels are quantized
+ * in the order of descending diag(H) (a zero diagonal counts as 1; equal values keep their
+ * original order), so the channels that see the largest activations are rounded first and are
+ * not used afterwards to absorb the error of the others.  The method is adadim_quantize_gptq
+ * applied to the reordered problem; every output is stored at the channel's ORIGINAL position,
+ * so the tensors have the same layout as without reordering:
+ *   per-IC  group parameters are taken from the current weights of the column being quantized,
+ *           as before; scales/zeros [out/g][in] stay contiguous (the point of Appendix A.1).
+ *   per-OC  "static groups" (Section 2.2): the parameters of every group of g consecutive
+ *           original columns are fixed from the original weights before anything is reordered
+ *           or updated (they equal adadim_quantize_rtn's per-OC parameters); a column is coded
+ *           with the parameters of the group it originally belongs to.
+ *   perm_out   optional device int32[in]: the order used (perm_out[i] = original index of the
+ *              i-th channel quantized).
+ *   The factor is always computed here (a factor of the unpermuted H does not apply).
+ *   Other arguments, shapes, workspace size (ADADIM_WS_GPTQ) and errors as adadim_quantize_gptq.
+ */
+ADADIM_API int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
+                         const float* H, int bits, int group, int dim,
+                         float percdamp, int blocksize,
+                         const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+                         double* gptq_loss, int32_t* perm_out, int* status_dev,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Reconstruction error of both quantized tensors and the selection (Section 3.3, Eq. 1;
  * Appendix B):  E_dim = || X (W - Q_dim)^T ||_F^2 = 1/2 trace((W - Q_dim) H (W - Q_dim)^T)
  * with the undamped H = 2 X^T X;  chosen = IC iff E_ic < E_oc (ties and NaN give OC, the

@@ -57,6 +57,9 @@ def lib():
         L.adadim_quantize_gptq.restype = C.c_int
         L.adadim_quantize_gptq.argtypes = [vp, C.c_int, i64, i64, i64, vp, vp, C.c_int, C.c_int, C.c_int, C.c_float,
                                            C.c_int, qp, qp, vp, vp, vp, sz, vp]
+        L.adadim_quantize_gptq_reordered.restype = C.c_int
+        L.adadim_quantize_gptq_reordered.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, C.c_int,
+                                                     C.c_float, C.c_int, qp, qp, vp, vp, vp, vp, sz, vp]
         L.adadim_score_select.restype = C.c_int
         L.adadim_score_select.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, qp, qp, vp, vp, vp, vp,
                                           sz, vp]
@@ -180,6 +183,35 @@ def quantize_gptq(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, dim: 
                                     status.data_ptr() if status is not None else None,
                                     workspace.data_ptr(), workspace.numel(), _stream())
     _check(rc, "adadim_quantize_gptq")
+    return q_oc, q_ic
+
+
+def quantize_gptq_reordered(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, dim: int = DIM_BOTH,
+                            percdamp: float = 0.01,
+                            q_oc: Optional[QTensor] = None, q_ic: Optional[QTensor] = None,
+                            loss: Optional[torch.Tensor] = None, perm: Optional[torch.Tensor] = None,
+                            status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+    """GPTQ with activation reordering (per-IC: dynamic groups; per-OC: static groups).
+    `perm`, if given, is an int32[in] device tensor that receives the column order."""
+    assert W.is_cuda and W.stride(1) == 1 and H.is_contiguous()
+    out, inp = W.shape
+    if dim != DIM_IC and q_oc is None:
+        q_oc = QTensor(out, inp, bits, group, DIM_OC, W.device)
+    if dim != DIM_OC and q_ic is None:
+        q_ic = QTensor(out, inp, bits, group, DIM_IC, W.device)
+    if workspace is None:
+        workspace = _ws(workspace_bytes(WS_GPTQ, out, inp, bits, group), W.device)
+    coc = q_oc.c() if q_oc is not None else None
+    cic = q_ic.c() if q_ic is not None else None
+    rc = lib().adadim_quantize_gptq_reordered(W.data_ptr(), _DT[W.dtype], out, inp, W.stride(0), H.data_ptr(),
+                                              bits, group, dim, percdamp, 128,
+                                              C.byref(coc) if coc is not None else None,
+                                              C.byref(cic) if cic is not None else None,
+                                              loss.data_ptr() if loss is not None else None,
+                                              perm.data_ptr() if perm is not None else None,
+                                              status.data_ptr() if status is not None else None,
+                                              workspace.data_ptr(), workspace.numel(), _stream())
+    _check(rc, "adadim_quantize_gptq_reordered")
     return q_oc, q_ic
 
 

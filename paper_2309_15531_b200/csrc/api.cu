@@ -14,11 +14,11 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
                  void* workspace, cudaStream_t st);
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
-                  cudaStream_t st);
+                  cudaStream_t st, const int* perm);
 size_t gptq_workspace_bytes(int64_t out, int64_t in);
 int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const float* U,
                 int bits, int group, int dim, float percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
-                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st);
+                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st, bool reorder, int* perm_out);
 
 namespace {
 
@@ -140,7 +140,7 @@ int adadim_cholesky_inverse_factor(const float* H, int64_t in, float percdamp, f
   if (workspace_bytes < factor_workspace_bytes(in)) return ADADIM_ERR_WORKSPACE;
   int rc = reset_status(status_dev, st);
   if (rc != ADADIM_OK) return rc;
-  return factor_launch(H, in, percdamp, U, status_dev, workspace, st);
+  return factor_launch(H, in, percdamp, U, status_dev, workspace, st, nullptr);
 }
 
 int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H,
@@ -167,7 +167,35 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
   rc = reset_status(status_dev, st);
   if (rc != ADADIM_OK) return rc;
   return gptq_launch(W, wdtype, out, in, ldw, H, U, bits, group, dim, percdamp, q_oc, q_ic, gptq_loss, status_dev,
-                     workspace, st);
+                     workspace, st, false, nullptr);
+}
+
+int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H,
+                                   int bits, int group, int dim, float percdamp, int blocksize,
+                                   const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* gptq_loss,
+                                   int32_t* perm_out, int* status_dev, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int rc = check_quant_params(bits, group);
+  if (rc != ADADIM_OK) return rc;
+  if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
+  if (blocksize != 128) return ADADIM_ERR_PARAM;
+  if (!(percdamp >= 0.0f) || !(percdamp < 1e6f)) return ADADIM_ERR_PARAM;
+  if (out < 0 || in < 0) return ADADIM_ERR_SHAPE;
+  if (out == 0 || in == 0) return ADADIM_OK;
+  rc = check_weight(W, wdtype, out, in, ldw);
+  if (rc != ADADIM_OK) return rc;
+  if (in % 128 != 0 || out % 128 != 0) return ADADIM_ERR_SHAPE;
+  if (H == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
+  if (!aligned16(H) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
+  const bool oc = dim != ADADIM_DIM_IC, ic = dim != ADADIM_DIM_OC;
+  if (oc && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
+  if (ic && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
+  if (workspace_bytes < gptq_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
+  rc = reset_status(status_dev, st);
+  if (rc != ADADIM_OK) return rc;
+  return gptq_launch(W, wdtype, out, in, ldw, H, nullptr, bits, group, dim, percdamp, q_oc, q_ic, gptq_loss,
+                     status_dev, workspace, st, true, perm_out);
 }
 
 int adadim_score_select(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, int bits,

@@ -178,15 +178,18 @@ damp_kernel(const float* __restrict__ H, int64_t n, double percdamp, double* sta
   if (threadIdx.x == 0) stats[0] = percdamp * red[0] / static_cast<double>(n);
 }
 
-// A[r][c] = Hd[n-1-r][n-1-c] on and below the diagonal, 0 above it
+// A[r][c] = Hd[p(n-1-r)][p(n-1-c)] on and below the diagonal, 0 above it; p is the column order
+// the caller quantizes in (identity when perm is null)
 __global__ void __launch_bounds__(256)
-build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ stats, double* __restrict__ A) {
+build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ stats, const int* __restrict__ perm,
+             double* __restrict__ A) {
   int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
   if (e >= n * n) return;
   int64_t r = e / n, c = e % n;
   double v = 0.0;
   if (r >= c) {
     int64_t i = n - 1 - r, j = n - 1 - c;
+    if (perm != nullptr) { i = perm[i]; j = perm[j]; }
     v = static_cast<double>(H[i * n + j]);
     if (i == j) {
       if (v == 0.0) v = 1.0;
@@ -572,7 +575,7 @@ FactorLayout factor_layout(int64_t n) {
 size_t factor_workspace_bytes(int64_t n) { return factor_layout(n).total; }
 
 int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
-                  cudaStream_t st) {
+                  cudaStream_t st, const int* perm) {
   FactorLayout Lo = factor_layout(n);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   double* A = reinterpret_cast<double*>(ws + Lo.a_off);
@@ -599,7 +602,7 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
   bool rest_pending = false;
 
   damp_kernel<<<1, 256, 0, st>>>(H, n, static_cast<double>(percdamp), stats);
-  build_kernel<<<eb, 256, 0, st>>>(H, n, stats, A);
+  build_kernel<<<eb, 256, 0, st>>>(H, n, stats, perm, A);
   ADADIM_CUDA_TRY(cudaEventRecord(ev_fork, st));
   ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_fork, 0));
   for (int g0 = 0; g0 < nb; g0 += kGroup) {

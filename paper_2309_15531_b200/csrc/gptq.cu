@@ -29,7 +29,7 @@ int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_
 
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
-                  cudaStream_t st);
+                  cudaStream_t st, const int* perm);
 
 namespace {
 
@@ -65,7 +65,111 @@ struct BlockArgs {
   int dim_of[2];             // grouping dimension of working copy d
   int64_t out, in;
   int i1;                    // first column of the block
+  // activation reordering (null / unused in the natural order): column i of the working copy is
+  // column perm[i] of W; per-OC parameters are fixed per original group beforehand
+  const int* perm;
+  const uint2* static_rec;   // [out][in/g]: {bits of 1/s (0: degenerate group), fp16 s | fp16 z << 16}
+  uint32_t* codes[2];        // where the block kernel writes codes (in working-copy column order)
 };
+
+// ---- activation reordering (paper Section 2.2, Appendix A.1) ---------------------------------
+// perm: input channels by descending diag(H) (a zero diagonal counts as 1, like the dead-column
+// fix), equal values in their original order; rank is its inverse.  Every channel counts the
+// channels that come before it: exact, deterministic, n^2 comparisons.
+__global__ void __launch_bounds__(256)
+order_kernel(const float* __restrict__ H, int64_t n, int* __restrict__ perm, int* __restrict__ rank) {
+  __shared__ float tile[256];
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  float di = 0.0f;
+  if (i < n) { di = H[i * n + i]; if (di == 0.0f) di = 1.0f; }
+  int before = 0;
+  for (int64_t j0 = 0; j0 < n; j0 += 256) {
+    const int64_t j = j0 + threadIdx.x;
+    float dj = 0.0f;
+    if (j < n) { dj = H[j * n + j]; if (dj == 0.0f) dj = 1.0f; }
+    __syncthreads();
+    tile[threadIdx.x] = dj;
+    __syncthreads();
+    const int lim = static_cast<int>(n - j0 < 256 ? n - j0 : 256);
+    for (int k = 0; k < lim; ++k) {
+      const float d = tile[k];
+      before += (d > di || (d == di && j0 + k < i)) ? 1 : 0;
+    }
+  }
+  if (i < n) { rank[i] = before; perm[before] = static_cast<int>(i); }
+}
+
+// Working copies in the quantization order: Wc[d][o][i] = W[o][perm[i]] (0 for dead columns).
+template <typename T>
+__global__ void __launch_bounds__(256)
+init_perm_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const float* __restrict__ H,
+                 const int* __restrict__ perm, int ndim, float* __restrict__ Wc) {
+  const int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (e >= out * in) return;
+  const int64_t o = e / in, c = perm[e % in];
+  float v = static_cast<float>(W[o * ldw + c]);
+  if (H[c * in + c] == 0.0f) v = 0.0f;
+  for (int d = 0; d < ndim; ++d) Wc[static_cast<int64_t>(d) * out * in + e] = v;
+}
+
+// Static per-OC groups: parameters of every group of g consecutive original columns, from the
+// original weights, before anything is reordered or updated.  One thread per (row, group).
+template <typename T, int BITS>
+__global__ void __launch_bounds__(256)
+static_params_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int group, adadim_qtensor q,
+                     uint2* __restrict__ rec) {
+  constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr float rcp_maxq = 1.0f / maxq;
+  const int64_t groups = in / group;
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (t >= out * groups) return;
+  const int64_t o = t / groups, g = t % groups;
+  const T* src = W + o * ldw + g * group;
+  float mn = 0.0f, mx = 0.0f;                     // 0 always lies inside [lo, hi]
+  for (int k = 0; k < group; k += 8) {
+    float v[8];
+    load8(src + k, v);
+#pragma unroll
+    for (int m = 0; m < 8; ++m) { mn = fminf(mn, v[m]); mx = fmaxf(mx, v[m]); }
+  }
+  const GroupParams gp = group_params(mn, mx, maxq, rcp_maxq);
+  const unsigned short sb = __half_as_ushort(__float2half_rn(gp.s)), zb = __half_as_ushort(__float2half_rn(gp.z));
+  q.scales[t] = sb;
+  q.zeros[t] = zb;
+  rec[t] = make_uint2(__float_as_uint(gp.rcp), static_cast<uint32_t>(sb) | (static_cast<uint32_t>(zb) << 16));
+}
+
+// Codes from working-copy column order back to the original columns: out word by out word,
+// code of original column c = code at position rank[c] of the row's temporary bitstream.
+template <int BITS>
+__global__ void __launch_bounds__(256)
+unpermute_codes_kernel(const uint32_t* __restrict__ tmp, const int* __restrict__ rank, int64_t out, int64_t in,
+                       uint32_t* __restrict__ codes) {
+  const int64_t chunks = in / 32;
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (t >= out * chunks) return;
+  const int64_t o = t / chunks, ch = t % chunks;
+  const uint32_t* row = tmp + o * (in * BITS / 32);
+  uint32_t wds[BITS] = {};
+#pragma unroll 4
+  for (int k = 0; k < 32; ++k) {
+    const int64_t bit = static_cast<int64_t>(rank[ch * 32 + k]) * BITS;
+    const int64_t wi = bit >> 5;
+    const int sh = static_cast<int>(bit & 31);
+    uint32_t v = row[wi] >> sh;
+    if (sh + BITS > 32) v |= row[wi + 1] << (32 - sh);
+    v &= (1u << BITS) - 1u;
+    const int ob = k * BITS, ow = ob >> 5, os = ob & 31;
+#pragma unroll
+    for (int m = 0; m < BITS; ++m) {
+      if (m == ow) wds[m] |= v << os;
+      if (m == ow + 1 && os + BITS > 32) wds[m] |= v >> (32 - os);
+    }
+  }
+  uint32_t* dst = codes + o * (in * BITS / 32) + ch * BITS;
+#pragma unroll
+  for (int m = 0; m < BITS; ++m) dst[m] = wds[m];
+}
 
 __device__ __forceinline__ int ordered_key(float v) {
   const int b = __float_as_int(v);
@@ -120,11 +224,22 @@ block_kernel(const BlockArgs a) {
     uint32_t cw[BITS] = {};
 #pragma unroll
     for (int k = 0; k < kSub; ++k) w[k] = wrow[cbase + k];
+    uint2 srec[kSub];                                // static per-OC records of these 32 columns
+    if (!is_ic && a.static_rec != nullptr) {
+#pragma unroll
+      for (int k = 0; k < kSub; ++k)
+        srec[k] = a.static_rec[row * (a.in / G) + a.perm[a.i1 + cbase + k] / G];
+    }
 
 #pragma unroll
     for (int ii = 0; ii < kSub; ++ii) {
       const int i = cbase + ii;                      // column inside the block
-      if (!is_ic) {
+      if (!is_ic && a.static_rec != nullptr) {       // per-OC, static groups: parameters fixed beforehand
+        const uint2 rec = srec[ii];
+        gp.rcp = __uint_as_float(rec.x);
+        gp.s = __half2float(__ushort_as_half(static_cast<unsigned short>(rec.y & 0xffffu)));
+        gp.z = __half2float(__ushort_as_half(static_cast<unsigned short>(rec.y >> 16)));
+      } else if (!is_ic) {
         if ((ii % G) == 0 && (cbase % G) == 0) {     // per-OC: parameters at the group's first column
           float mn = w[ii], mx = w[ii];
           if (G == kSub) {
@@ -176,7 +291,7 @@ block_kernel(const BlockArgs a) {
       for (int jj = ii + 1; jj < kSub; ++jj) w[jj] = fmaf(-e, urow[jj], w[jj]);
     }
     // codes of these 32 columns: BITS whole words of this row's bitstream
-    uint32_t* cdst = q.codes + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
+    uint32_t* cdst = a.codes[d] + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
 #pragma unroll
     for (int k = 0; k < BITS; ++k) cdst[k] = cw[k];
     // lazy update of the block's later columns with this sub-block's 32 errors
@@ -229,7 +344,8 @@ block_kernel(const BlockArgs a) {
   }
   if (is_ic) {
     for (int e = tid; e < NG * kBlk; e += kBlk) {
-      int64_t idx = (row0 / G + e / kBlk) * a.in + a.i1 + (e % kBlk);
+      const int wc = a.i1 + (e % kBlk);               // working-copy column -> original column
+      int64_t idx = (row0 / G + e / kBlk) * a.in + (a.perm != nullptr ? a.perm[wc] : wc);
       q.scales[idx] = Ss[e];
       q.zeros[idx] = Zs[e];
     }
@@ -264,7 +380,10 @@ int block_launch(const BlockArgs& a, int slabs, int ndim, cudaStream_t st) {
   return ADADIM_OK;
 }
 
-struct GptqLayout { size_t wc_off, err_off, err_piece, loss_off, up_off, up_piece, u_off, factor_off, total; };
+struct GptqLayout {
+  size_t wc_off, err_off, err_piece, loss_off, up_off, up_piece, u_off, factor_off;
+  size_t perm_off, rank_off, rec_off, tmp_off, tmp_piece, total;     // used by the reordered variant only
+};
 GptqLayout gptq_layout(int64_t out, int64_t in) {
   GptqLayout L;
   size_t off = 0;
@@ -276,6 +395,11 @@ GptqLayout gptq_layout(int64_t out, int64_t in) {
   L.loss_off = off;   off += round_up(static_cast<size_t>(2) * (out / kBlk + 1) * 8, 256);
   L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 4, 256);
   L.factor_off = off; off += factor_workspace_bytes(in);
+  L.perm_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
+  L.rank_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
+  L.rec_off = off;    off += round_up(static_cast<size_t>(out) * (in / 32) * 8, 256);     // g >= 32
+  L.tmp_piece = round_up(static_cast<size_t>(out) * in / 2, 256);                          // bits <= 4
+  L.tmp_off = off;    off += 2 * L.tmp_piece;
   L.total = off;
   return L;
 }
@@ -286,7 +410,7 @@ size_t gptq_workspace_bytes(int64_t out, int64_t in) { return gptq_layout(out, i
 
 int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const float* U_in,
                 int bits, int group, int dim, float percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
-                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st) {
+                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st, bool reorder, int* perm_out) {
   GptqLayout L = gptq_layout(out, in);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   BlockArgs a = {};
@@ -305,10 +429,35 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   if (dim == ADADIM_DIM_OC || dim == ADADIM_DIM_BOTH) { a.q[ndim] = *q_oc; a.dim_of[ndim] = ADADIM_DIM_OC; ++ndim; }
   if (dim == ADADIM_DIM_IC || dim == ADADIM_DIM_BOTH) { a.q[ndim] = *q_ic; a.dim_of[ndim] = ADADIM_DIM_IC; ++ndim; }
 
+  int* perm = nullptr;
+  int* rank = nullptr;
+  for (int d = 0; d < ndim; ++d) a.codes[d] = a.q[d].codes;
+  if (reorder) {
+    perm = reinterpret_cast<int*>(ws + L.perm_off);
+    rank = reinterpret_cast<int*>(ws + L.rank_off);
+    order_kernel<<<static_cast<unsigned>((in + 255) / 256), 256, 0, st>>>(H, in, perm, rank);
+    if (perm_out != nullptr)
+      ADADIM_CUDA_TRY(cudaMemcpyAsync(perm_out, perm, static_cast<size_t>(in) * 4, cudaMemcpyDeviceToDevice, st));
+    a.perm = perm;
+    for (int d = 0; d < ndim; ++d) a.codes[d] = reinterpret_cast<uint32_t*>(ws + L.tmp_off + d * L.tmp_piece);
+    if (a.dim_of[0] == ADADIM_DIM_OC) {              // static groups for the per-OC copy (always copy 0)
+      uint2* rec = reinterpret_cast<uint2*>(ws + L.rec_off);
+      const unsigned sb = static_cast<unsigned>((out * (in / group) + 255) / 256);
+      if (wdtype == ADADIM_F16) {
+        if (bits == 3) static_params_kernel<__half, 3><<<sb, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, group, a.q[0], rec);
+        else static_params_kernel<__half, 4><<<sb, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, group, a.q[0], rec);
+      } else {
+        if (bits == 3) static_params_kernel<float, 3><<<sb, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, group, a.q[0], rec);
+        else static_params_kernel<float, 4><<<sb, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, group, a.q[0], rec);
+      }
+      a.static_rec = rec;
+    }
+  }
+
   const float* U = U_in;
-  if (U == nullptr) {
+  if (U == nullptr || reorder) {                     // a caller's factor belongs to the natural order
     float* Uw = reinterpret_cast<float*>(ws + L.u_off);
-    int rc = factor_launch(H, in, percdamp, Uw, status_dev, ws + L.factor_off, st);
+    int rc = factor_launch(H, in, percdamp, Uw, status_dev, ws + L.factor_off, st, perm);
     if (rc != ADADIM_OK) return rc;
     U = Uw;
   }
@@ -317,9 +466,15 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
                           const_cast<__nv_bfloat16*>(up[2]), st);
   if (rc0 != ADADIM_OK) return rc0;
 
-  const unsigned ib = static_cast<unsigned>((out * in / 8 + 255) / 256);
-  if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, ndim, a.Wc);
-  else init_kernel<<<ib, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, H, ndim, a.Wc);
+  if (reorder) {
+    const unsigned pb = static_cast<unsigned>((out * in + 255) / 256);
+    if (wdtype == ADADIM_F16) init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, perm, ndim, a.Wc);
+    else init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, H, perm, ndim, a.Wc);
+  } else {
+    const unsigned ib = static_cast<unsigned>((out * in / 8 + 255) / 256);
+    if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, ndim, a.Wc);
+    else init_kernel<<<ib, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, H, ndim, a.Wc);
+  }
   ADADIM_CUDA_TRY(cudaMemsetAsync(a.loss_part, 0, static_cast<size_t>(2) * (out / kBlk + 1) * 8, st));
 
   const int slabs = static_cast<int>(out / kBlk);
@@ -388,6 +543,13 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   cudaStreamDestroy(chain);
   cudaStreamDestroy(side);
   for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k];
+  if (reorder) {
+    const unsigned ub = static_cast<unsigned>((out * (in / 32) + 255) / 256);
+    for (int d = 0; d < ndim; ++d) {
+      if (bits == 3) unpermute_codes_kernel<3><<<ub, 256, 0, st>>>(a.codes[d], rank, out, in, a.q[d].codes);
+      else unpermute_codes_kernel<4><<<ub, 256, 0, st>>>(a.codes[d], rank, out, in, a.q[d].codes);
+    }
+  }
   if (gptq_loss != nullptr) loss_kernel<<<1, 32, 0, st>>>(a.loss_part, ndim, slabs, a, gptq_loss);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
