@@ -361,6 +361,14 @@ def gptq_ada(W, H, bits, group, percdamp=0.01):
     return best, err, quantize_gptq(W, H, bits, group, best, percdamp)
 
 
+def gptq_ada_reordered(W, H, bits, group, percdamp=0.01):
+    """The paper's final GPTQ design (Section 4.1; Appendix A.1): the dimension is chosen with RTN,
+    then GPTQ runs in it with activation reordering: static groups if per-OC was chosen, plain
+    reordering if per-IC was."""
+    best, err, _ = rtn_ada(W, H, bits, group)
+    return best, err, quantize_gptq_reordered(W, H, bits, group, best, percdamp, static_groups=(best == "oc"))
+
+
 def gptq_both(W, H, bits, group, percdamp=0.01):
     """GPTQ in both dimensions, scored with the undamped H, lower error kept."""
     Hd, dead = damped_hessian(H, percdamp)

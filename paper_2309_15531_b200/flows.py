@@ -30,6 +30,16 @@ def gptq_ada(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, percdamp: 
     return dim, err, (q_oc if dim == B.DIM_OC else q_ic)
 
 
+def gptq_ada_reordered(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, percdamp: float = 0.01,
+                       status: Optional[torch.Tensor] = None):
+    """The paper's final GPTQ design (Section 4.1, Appendix A.1): choose the dimension with RTN,
+    then GPTQ in it with activation reordering (static groups when per-OC was chosen).
+    Returns (chosen dim, RTN errors, quantized tensor of the chosen dimension)."""
+    dim, err, _ = rtn_ada(W, H, bits, group, status)
+    q_oc, q_ic = B.quantize_gptq_reordered(W, H, bits, group, dim, percdamp, status=status)
+    return dim, err, (q_oc if dim == B.DIM_OC else q_ic)
+
+
 def gptq_both(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, percdamp: float = 0.01,
               U: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
     """GPTQ in both dimensions, scored with the undamped H, lower error kept.

@@ -110,3 +110,20 @@ def test_reordered_result_beats_rtn_on_correlated_activations():
     torch.cuda.synchronize()
     print(f"E_ic reordered {err_r[1].item():.6e}  natural {err_p[1].item():.6e}  rtn {err_t[1].item():.6e}")
     assert err_r[1].item() < err_t[1].item() and err_p[1].item() < err_t[1].item()
+
+
+def test_reordered_flow_matches_the_oracle_flow():
+    from paper_2309_15531_b200 import flows
+    W = I.make_weight(I.WeightSpec(256, 256, "f16", 0.02, 0.0, seed=69), "cuda")
+    X = I.make_calib(I.CalibSpec(2048, 256, "bf16", "normal", 3, 50.0, 100.0, seed=70), "cuda")
+    W[:, :8] *= 0.1                                        # make the dimensions differ clearly
+    Wn = to_np(W).astype(np.float32)
+    Hn = O.hessian(to_np(X)).astype(np.float32)
+    dim, err, q = flows.gptq_ada_reordered(W, torch.as_tensor(Hn, device="cuda"), 3, 128)
+    torch.cuda.synchronize()
+    best, ref_err, ref = O.gptq_ada_reordered(Wn, Hn.astype(np.float64), 3, 128)
+    assert B.DIM_NAMES[dim] == best
+    assert err[0].item() == pytest.approx(ref_err["oc"], rel=1e-3) and err[1].item() == pytest.approx(ref_err["ic"], rel=1e-3)
+    codes, _, _ = q_to_np(q)
+    frac, lvl = code_mismatch(codes, ref["codes"])
+    assert frac <= 1e-3 and lvl <= 1

@@ -317,3 +317,12 @@ def test_reordered_loss_identity_and_static_parameters(dim):
         assert np.array_equal(r["zeros"].view(np.uint16), t["zeros"].view(np.uint16))
     with pytest.raises(ValueError):
         O.quantize_gptq_reordered(W, H, 3, 32, "oc", static_groups=False)
+
+
+def test_reordered_flow_uses_the_rtn_choice():
+    W, X = _layer(128, 128, 400, outliers=(5, 77), scale=60.0)
+    H = O.hessian(X)
+    best, err, r = O.gptq_ada_reordered(W, H, 3, 128)
+    assert best == O.rtn_ada(W, H, 3, 128)[0]
+    ref = O.quantize_gptq_reordered(W, H, 3, 128, best, static_groups=(best == "oc"))
+    assert np.array_equal(r["codes"], ref["codes"])
