@@ -199,6 +199,43 @@ build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ 
   A[e] = v;
 }
 
+// One merge level of the in-block inverse (shared memory, 256 threads): for every pair of
+// adjacent SZ x SZ inverted diagonal blocks XA, XB with the block C of the factor between them,
+//   T = C XA,   C <- -XB T.
+// A thread owns SZ/8 elements, a warp one row of T at a time (for SZ = 32), so the first operand
+// is a broadcast and the second is read along a row.  M is zero above the diagonal, which lets
+// both sums run over the whole range with compile-time bounds.
+template <int SZ>
+__device__ __forceinline__ void merge_level(double (*M)[kNB + 1], double (*T)[kNB / 2 + 1], int tid) {
+  constexpr int PER = SZ / 8;
+  int gi[PER], jj[PER], a0[PER];
+  double acc[PER];
+#pragma unroll
+  for (int u = 0; u < PER; ++u) {
+    const int e = tid + 256 * u;
+    gi[u] = e / SZ;
+    jj[u] = e % SZ;
+    a0[u] = (gi[u] / SZ) * 2 * SZ;
+    acc[u] = 0.0;
+  }
+#pragma unroll
+  for (int m = 0; m < SZ; ++m)
+#pragma unroll
+    for (int u = 0; u < PER; ++u)
+      acc[u] = fma(M[a0[u] + SZ + gi[u] % SZ][a0[u] + m], M[a0[u] + m][a0[u] + jj[u]], acc[u]);
+#pragma unroll
+  for (int u = 0; u < PER; ++u) { T[gi[u]][jj[u]] = acc[u]; acc[u] = 0.0; }
+  __syncthreads();
+#pragma unroll
+  for (int m = 0; m < SZ; ++m)
+#pragma unroll
+    for (int u = 0; u < PER; ++u)
+      acc[u] = fma(M[a0[u] + SZ + gi[u] % SZ][a0[u] + SZ + m], T[(gi[u] / SZ) * SZ + m][jj[u]], acc[u]);
+#pragma unroll
+  for (int u = 0; u < PER; ++u) M[a0[u] + SZ + gi[u] % SZ][a0[u] + jj[u]] = -acc[u];
+  __syncthreads();
+}
+
 // ---- factorization -------------------------------------------------------------------------
 // Diagonal block k: in-place Cholesky of the 64 x 64 block and its triangular inverse -> dinv[k].
 // The block is worked in eight sub-panels of eight columns, right-looking inside shared memory:
@@ -217,7 +254,19 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
   __shared__ double rdiag[kNB];          // 1 / L[j][j]
   const int tid = threadIdx.x;
   double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
-  for (int e = tid; e < kNB * kNB; e += 256) M[e >> 6][e & 63] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
+  {
+    double v[kNB * kNB / 256];                         // all loads in flight before the first store
+#pragma unroll
+    for (int u = 0; u < kNB * kNB / 256; ++u) {
+      const int e = tid + 256 * u;
+      v[u] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
+    }
+#pragma unroll
+    for (int u = 0; u < kNB * kNB / 256; ++u) {
+      const int e = tid + 256 * u;
+      M[e >> 6][e & 63] = v[u];
+    }
+  }
   __syncthreads();
 
 #pragma unroll 1
@@ -250,13 +299,12 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
 #pragma unroll
           for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
       }
-      if (row < kNB) {
+      if (row < kNB) {                               // x D^T = a by substitution, finished entries pushed forward
 #pragma unroll
         for (int c = 0; c < kSub; ++c) {
-          double sacc = x[c];
+          x[c] *= rinv[c];
 #pragma unroll
-          for (int m = 0; m < c; ++m) sacc = fma(-x[m], d[c][m], sacc);
-          x[c] = sacc * rinv[c];
+          for (int c2 = c + 1; c2 < kSub; ++c2) x[c2] = fma(-x[c], d[c2][c], x[c2]);
         }
       }
     }
@@ -332,50 +380,9 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
     }
   }
   __syncthreads();
-#pragma unroll 1
-  for (int sz = kSub; sz < kNB; sz *= 2) {
-    // pair p: A part rows/cols [p*2sz, p*2sz+sz), B part the next sz; T[p*sz + i][j] = (C XA)[i][j].
-    // A thread works on up to four elements at once (32*sz/256 = sz/8 <= 4) so that the dependent
-    // chains of multiply-adds overlap; terms outside the triangles are zeros in M.
-    const int per = sz / 8;                            // elements per thread: 1, 2, 4
-    {
-      int gi[4], jj[4];
-      double sacc[4] = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll
-      for (int u = 0; u < 4; ++u) { const int e = tid + 256 * (u < per ? u : 0); gi[u] = e / sz; jj[u] = e % sz; }
-      for (int m = 0; m < sz; ++m) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int p = gi[u] / sz, i = gi[u] % sz, a0 = p * 2 * sz, b0 = a0 + sz;
-          sacc[u] = fma(M[b0 + i][a0 + m], M[a0 + m][a0 + jj[u]], sacc[u]);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) if (u < per) T[gi[u]][jj[u]] = sacc[u];
-    }
-    __syncthreads();
-    {
-      int gi[4], jj[4];
-      double sacc[4] = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll
-      for (int u = 0; u < 4; ++u) { const int e = tid + 256 * (u < per ? u : 0); gi[u] = e / sz; jj[u] = e % sz; }
-      for (int m = 0; m < sz; ++m) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int p = gi[u] / sz, i = gi[u] % sz, b0 = p * 2 * sz + sz;
-          sacc[u] = fma(M[b0 + i][b0 + m], T[p * sz + m][jj[u]], sacc[u]);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (u < per) {
-          const int p = gi[u] / sz, i = gi[u] % sz, a0 = p * 2 * sz, b0 = a0 + sz;
-          M[b0 + i][a0 + jj[u]] = -sacc[u];
-        }
-      }
-    }
-    __syncthreads();
-  }
+  merge_level<8>(M, T, tid);
+  merge_level<16>(M, T, tid);
+  merge_level<32>(M, T, tid);
   double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
   for (int e = tid; e < kNB * kNB; e += 256) {
     const int r = e >> 6, c = e & 63;
