@@ -5,7 +5,7 @@
 // triangle; then U = P L^-1 P, because Hd = (P L P)(P L P)^T with P L P upper triangular and
 // Hd^-1 = (P L^-1 P)^T (P L^-1 P).  This needs one factorization and one triangular inverse
 // instead of a factorization, a full inverse and a second factorization.  All arithmetic is
-// binary64 on the CUDA cores (the factor decides GPTQ's rounding, so it is kept well inside
+// binary64, the large products on the fp64 matrix instruction (the factor decides GPTQ's rounding, so it is kept well inside
 // the fp32 precision of U); U is rounded to fp32 on output.
 //
 //   factorization : 64-column panels (diagonal block on one CTA, then the panel below it
@@ -29,37 +29,42 @@ constexpr int kGroup = 4;   // panels per rank-256 update
 __host__ __device__ __forceinline__ int64_t mn64(int64_t a, int64_t b) { return a < b ? a : b; }
 
 // ---- 64 x 64 output tile product, 256 threads, 4 x 4 outputs per thread --------------------
-// acc += A[64 x K] * B, A row-major with leading dimension lda;
-// B_T: B is given as [64 cols][K] row-major (product with the transpose), else as [K][64 cols].
+// acc += A[64 x 64] * B, A row-major with leading dimension lda;
+// B_T: B is given as [64 cols][64] row-major (product with the transpose), else as [64][64 cols].
+// These tiles sit on the factorization's critical chain, so every global load of the tile is
+// issued before the first one is used: one memory latency per tile instead of one per slab.
 template <bool B_T>
 __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64_t lda, const double* __restrict__ B,
                                              int64_t ldb, int K, double (&acc)[4][4], double (*sa)[kNB + 2],
                                              double (*sb)[kNB + 2]) {
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  for (int k0 = 0; k0 < K; k0 += 16) {
-    {
-      const int r = threadIdx.x >> 2, kq = (threadIdx.x & 3) * 4;
-      const double2* src = reinterpret_cast<const double2*>(A + static_cast<int64_t>(r) * lda + k0 + kq);
-      double2 v0 = src[0], v1 = src[1];
-      sa[kq + 0][r] = v0.x; sa[kq + 1][r] = v0.y; sa[kq + 2][r] = v1.x; sa[kq + 3][r] = v1.y;
-    }
+  constexpr int kSlabs = kNB / 16;
+  double2 av[kSlabs][2], bv[kSlabs][2];
+  const int r = threadIdx.x >> 2, kq = (threadIdx.x & 3) * 4;          // loader: row (or column of B^T), first k of four
+  const int kk = threadIdx.x >> 4, nq = (threadIdx.x & 15) * 4;        // loader of a non-transposed B: k row, first column
+#pragma unroll
+  for (int sl = 0; sl < kSlabs; ++sl) {
+    const double2* asrc = reinterpret_cast<const double2*>(A + static_cast<int64_t>(r) * lda + sl * 16 + kq);
+    av[sl][0] = asrc[0]; av[sl][1] = asrc[1];
+    const double2* bsrc = B_T ? reinterpret_cast<const double2*>(B + static_cast<int64_t>(r) * ldb + sl * 16 + kq)
+                              : reinterpret_cast<const double2*>(B + static_cast<int64_t>(sl * 16 + kk) * ldb + nq);
+    bv[sl][0] = bsrc[0]; bv[sl][1] = bsrc[1];
+  }
+  (void)K;
+#pragma unroll
+  for (int sl = 0; sl < kSlabs; ++sl) {
+    sa[kq + 0][r] = av[sl][0].x; sa[kq + 1][r] = av[sl][0].y; sa[kq + 2][r] = av[sl][1].x; sa[kq + 3][r] = av[sl][1].y;
     if (B_T) {
-      const int r = threadIdx.x >> 2, kq = (threadIdx.x & 3) * 4;
-      const double2* src = reinterpret_cast<const double2*>(B + static_cast<int64_t>(r) * ldb + k0 + kq);
-      double2 v0 = src[0], v1 = src[1];
-      sb[kq + 0][r] = v0.x; sb[kq + 1][r] = v0.y; sb[kq + 2][r] = v1.x; sb[kq + 3][r] = v1.y;
+      sb[kq + 0][r] = bv[sl][0].x; sb[kq + 1][r] = bv[sl][0].y; sb[kq + 2][r] = bv[sl][1].x; sb[kq + 3][r] = bv[sl][1].y;
     } else {
-      const int kk = threadIdx.x >> 4, nq = (threadIdx.x & 15) * 4;
-      const double2* src = reinterpret_cast<const double2*>(B + static_cast<int64_t>(k0 + kk) * ldb + nq);
-      double2 v0 = src[0], v1 = src[1];
-      sb[kk][nq + 0] = v0.x; sb[kk][nq + 1] = v0.y; sb[kk][nq + 2] = v1.x; sb[kk][nq + 3] = v1.y;
+      sb[kk][nq + 0] = bv[sl][0].x; sb[kk][nq + 1] = bv[sl][0].y; sb[kk][nq + 2] = bv[sl][1].x; sb[kk][nq + 3] = bv[sl][1].y;
     }
     __syncthreads();
 #pragma unroll
-    for (int kk = 0; kk < 16; ++kk) {
+    for (int k2 = 0; k2 < 16; ++k2) {
       double a[4], b[4];
 #pragma unroll
-      for (int m = 0; m < 4; ++m) { a[m] = sa[kk][ty * 4 + m]; b[m] = sb[kk][tx * 4 + m]; }
+      for (int m = 0; m < 4; ++m) { a[m] = sa[k2][ty * 4 + m]; b[m] = sb[k2][tx * 4 + m]; }
 #pragma unroll
       for (int m = 0; m < 4; ++m)
 #pragma unroll
@@ -73,23 +78,35 @@ __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64
   __shared__ double sa[16][kNB + 2];   \
   __shared__ double sb[16][kNB + 2];
 
-// ---- 128 x 64 output tile product, 256 threads, 8 x 4 outputs per thread -------------------
-// Output rows of a thread: ty*4 + {0..3} and 64 + ty*4 + {0..3}; columns tx*4 + {0..3}.
-// Rows >= a_rows (64 or 128) of A are not read (treated as zero).  K is a multiple of 8.
-// Shared-memory slabs are double-buffered; the slab after the next one is already on its way
-// from global memory into registers while the current one is multiplied, and two CTAs share an
-// SM, so global latency is covered.
+// ---- 128 x 64 output tile product on the fp64 tensor-core path, 256 threads ----------------
+// Each of the eight warps owns a 32 x 32 piece of the tile as 4 x 4 fragments of the 8 x 8 x 4
+// fp64 matrix instruction (full fp64 multiply-add rate with an eighth of the instruction issue and
+// a fraction of the shared-memory traffic of scalar multiply-adds, which were bound by shared-memory
+// bandwidth here).  Rows >= a_rows (64 or 128) of A are not read (treated as zero).  K is a
+// multiple of 8.  Shared-memory slabs are double-buffered; the slab after the next one is already
+// on its way from global memory into registers while the current one is multiplied, and two CTAs
+// share an SM, so global latency is covered.  The row pitches are 8 mod 16 doubles: the 4 k-rows
+// x 8 columns of a fragment load then fall on distinct banks.
 constexpr int kT = 128, kTN = 64, kBK = 8;
 struct TileSmem {
-  double a[2][kBK][kT + 4];
-  double b[2][kBK][kTN + 4];
+  double a[2][kBK][kT + 8];
+  double b[2][kBK][kTN + 8];
 };
 
+__device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
+}
+
+// acc[i][j] is the fragment at rows 8 i, columns 8 j of the warp's piece: this lane holds row
+// lane / 4 and columns 2 (lane % 4), 2 (lane % 4) + 1 of it.
 template <bool B_T>
 __device__ __forceinline__ void product_tile(const double* __restrict__ A, int64_t lda, int a_rows,
                                              const double* __restrict__ B, int64_t ldb, int K,
-                                             double (&acc)[8][4], TileSmem& sm) {
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+                                             double (&acc)[4][4][2], TileSmem& sm) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 3) * 32, wn = (warp >> 2) * 32;
+  const int fk = lane & 3, fr = lane >> 2;                      // fragment coordinates of this lane
   const int ar = tid >> 1, akq = (tid & 1) * 4;                 // A loader: row, first k of four
   const int br = tid >> 2, bkq = (tid & 3) * 2;                 // B loader (transposed): column, first k of two
   const int bkk = tid >> 5, bnq = (tid & 31) * 2;               // B loader (not transposed): k row, first col of two
@@ -114,19 +131,17 @@ __device__ __forceinline__ void product_tile(const double* __restrict__ A, int64
   };
   auto multiply = [&](int buf) {
 #pragma unroll
-    for (int kk = 0; kk < kBK; ++kk) {
-      __align__(16) double a[8];
-      __align__(16) double b[4];
-      *reinterpret_cast<double2*>(a + 0) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4]);
-      *reinterpret_cast<double2*>(a + 2) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][ty * 4 + 2]);
-      *reinterpret_cast<double2*>(a + 4) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4]);
-      *reinterpret_cast<double2*>(a + 6) = *reinterpret_cast<const double2*>(&sm.a[buf][kk][64 + ty * 4 + 2]);
-      *reinterpret_cast<double2*>(b + 0) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][tx * 4]);
-      *reinterpret_cast<double2*>(b + 2) = *reinterpret_cast<const double2*>(&sm.b[buf][kk][tx * 4 + 2]);
+    for (int ks = 0; ks < kBK; ks += 4) {
+      double af[4], bf[4];
 #pragma unroll
-      for (int m = 0; m < 8; ++m)
+      for (int i = 0; i < 4; ++i) {
+        af[i] = sm.a[buf][ks + fk][wm + 8 * i + fr];
+        bf[i] = sm.b[buf][ks + fk][wn + 8 * i + fr];
+      }
 #pragma unroll
-        for (int n = 0; n < 4; ++n) acc[m][n] = fma(a[m], b[n], acc[m][n]);
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mma_f64(acc[i][j], af[i], bf[j]);
     }
   };
 
@@ -151,12 +166,15 @@ __device__ __forceinline__ void product_tile(const double* __restrict__ A, int64
   }
 }
 
-// Applies f(row, first column, values of 4 consecutive columns) to a thread's 8 x 4 outputs.
+// Applies f(row, first column, values of 2 consecutive columns) to a thread's outputs.
 template <typename F>
-__device__ __forceinline__ void for_each_quad(double (&acc)[8][4], F f) {
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+__device__ __forceinline__ void for_each_pair(double (&acc)[4][4][2], F f) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int wm = (warp & 3) * 32, wn = (warp >> 2) * 32;
 #pragma unroll
-  for (int m = 0; m < 8; ++m) f((m < 4 ? 0 : 64) + ty * 4 + (m & 3), tx * 4, &acc[m][0]);
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) f(wm + 8 * i + (lane >> 2), wn + 8 * j + 2 * (lane & 3), acc[i][j]);
 }
 
 // ---- set-up --------------------------------------------------------------------------------
@@ -452,15 +470,15 @@ rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int
   const int64_t ri = e + static_cast<int64_t>(ti) * kT, rj = e + static_cast<int64_t>(cj) * kTN;
   if (rj >= n) return;
   const int vr = static_cast<int>(mn64(kT, n - ri));
-  double acc[8][4] = {};
+  double acc[4][4][2] = {};
   product_tile<true>(A + ri * n + j0, n, vr, A + rj * n + j0, n, kw, acc, sm);
   const int skip_rows = cj == 2 * ti + 1 ? 64 : 0;
-  for_each_quad(acc, [&](int r, int c4, const double* v) {
+  for_each_pair(acc, [&](int r, int c2, const double* v) {
     if (r >= vr || r < skip_rows) return;
-    double2* p = reinterpret_cast<double2*>(A + (ri + r) * n + rj + c4);
-    double2 u0 = p[0], u1 = p[1];
-    u0.x -= v[0]; u0.y -= v[1]; u1.x -= v[2]; u1.y -= v[3];
-    p[0] = u0; p[1] = u1;
+    double2* p = reinterpret_cast<double2*>(A + (ri + r) * n + rj + c2);
+    double2 u = *p;
+    u.x -= v[0]; u.y -= v[1];
+    *p = u;
   });
 }
 
@@ -520,15 +538,13 @@ merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __rest
   if (static_cast<int64_t>(r) * kT >= sB) return;
   const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
   const int64_t m0 = static_cast<int64_t>(c) * kTN;
-  double acc[8][4] = {};
+  double acc[4][4][2] = {};
   product_tile<false>(A + (b0 + static_cast<int64_t>(r) * kT) * n + a0 + m0, n, vr, A + (a0 + m0) * n + a0 + m0, n,
                       static_cast<int>(s - m0), acc, sm);
   double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kT * s + m0;
-  for_each_quad(acc, [&](int rr, int c4, const double* v) {
+  for_each_pair(acc, [&](int rr, int c2, const double* v) {
     if (rr >= vr) return;
-    double2* p = reinterpret_cast<double2*>(t + static_cast<int64_t>(rr) * s + c4);
-    p[0] = make_double2(v[0], v[1]);
-    p[1] = make_double2(v[2], v[3]);
+    *reinterpret_cast<double2*>(t + static_cast<int64_t>(rr) * s + c2) = make_double2(v[0], v[1]);
   });
 }
 __global__ void __launch_bounds__(256, 2)
@@ -544,15 +560,13 @@ merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __rest
   const int64_t row0 = b0 + static_cast<int64_t>(r) * kT;
   const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
   const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kT, sB));
-  double acc[8][4] = {};
+  double acc[4][4][2] = {};
   product_tile<false>(A + row0 * n + b0, n, vr, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kTN,
                       s, K, acc, sm);
   double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kTN;
-  for_each_quad(acc, [&](int rr, int c4, const double* v) {
+  for_each_pair(acc, [&](int rr, int c2, const double* v) {
     if (rr >= vr) return;
-    double2* p = reinterpret_cast<double2*>(dst + static_cast<int64_t>(rr) * n + c4);
-    p[0] = make_double2(-v[0], -v[1]);
-    p[1] = make_double2(-v[2], -v[3]);
+    *reinterpret_cast<double2*>(dst + static_cast<int64_t>(rr) * n + c2) = make_double2(-v[0], -v[1]);
   });
 }
 
