@@ -17,7 +17,7 @@
 namespace adadim {
 
 struct TrailPlan {
-  CUtensorMap e[3], u[3];
+  CUtensorMap e[3], u[3], w;
   float* Wc;
   int64_t rows_total, in;
   int sm_count;

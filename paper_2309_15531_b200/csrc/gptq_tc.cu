@@ -30,7 +30,8 @@ constexpr int kTileN = 128;
 constexpr uint32_t kBPiece = kTileN * 32 * 2;       // one U piece, 32 k-rows x 128 columns: 8 KB
 constexpr uint32_t kBStage = 3 * kBPiece;           // 24 KB
 constexpr int kBStages = 4;
-constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 1024 + 256;
+constexpr uint32_t kOutChunk = 32 * 32 * 4;          // one epilogue warp's staging tile: 32 rows x 32 fp32 columns
+constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 8 * kOutChunk + 1024 + 256;
 
 struct TrailParams {
   float* Wc;            // [rows_total][in] stacked working weights
@@ -46,12 +47,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ CUtensorMap tmE1,
              const __grid_constant__ CUtensorMap tmE2, const __grid_constant__ CUtensorMap tmU0,
              const __grid_constant__ CUtensorMap tmU1, const __grid_constant__ CUtensorMap tmU2,
+             const __grid_constant__ CUtensorMap tmW,
              const TrailParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_smem = smem;
   uint8_t* b_smem = smem + kABytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + kBStages * kBStage);
+  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][32 rows][128 B], 128-byte swizzle
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 8 * kOutChunk);
   uint64_t* a_full = bars;
   uint64_t* b_full = bars + 1;                      // [kBStages]
   uint64_t* b_empty = b_full + kBStages;            // [kBStages]
@@ -166,18 +169,16 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
       }
     }
   } else {
-    // two warps per TMEM lane quadrant, each taking one 64-column half of every tile
+    // Two warps per TMEM lane quadrant, each taking one 64-column half of every tile.  W is never
+    // read here: the negated product goes to a staging tile in shared memory and from there into
+    // W as an element-wise add done by the memory system (W + (-p) is the same binary32 operation
+    // as W - p), 32 rows x 32 columns at a time, so the epilogue only issues writes.
     const int q = warp & 3, half = (warp - 2) >> 2;
     uint32_t acc_phase[2] = {0, 0};
-    float* wrow = p.Wc + (static_cast<int64_t>(mrow) + q * 32 + lane) * p.in + half * 64;
+    uint8_t* stage_tile = out_smem + (warp - 2) * kOutChunk;
+    uint8_t* my_row = stage_tile + lane * 128;        // this lane's row of the staging tile
     for (int t = t0; t < t1; ++t) {
       const int buf = (t - t0) & 1;
-      // The tile's slice of W does not depend on the MMAs: fetch it while they run.
-      // (in % 128 == 0 and c0 % 128 == 0, so every tile lies wholly inside the matrix.)
-      float4* w4 = reinterpret_cast<float4*>(wrow + p.c0 + static_cast<int64_t>(t) * kTileN);
-      float4 w[16];
-#pragma unroll
-      for (int k = 0; k < 16; ++k) w[k] = w4[k];
       if (!ptx::mbar_wait(&acc_full[buf], acc_phase[buf], dead, p.status_dev)) break;
       ptx::tc_fence_after_sync();
 #pragma unroll
@@ -186,12 +187,20 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + half * 64 + c * 32;
         ptx::tmem_ld32(taddr, v);
         ptx::tmem_ld32(taddr + kTileN, v2);
+        if (lane == 0) ptx::bulk_wait_read();         // the previous add has finished reading the staging tile
+        __syncwarp();
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          float4 x = w[c * 8 + k];
-          x.x -= v[4 * k] + v2[4 * k];         x.y -= v[4 * k + 1] + v2[4 * k + 1];
-          x.z -= v[4 * k + 2] + v2[4 * k + 2]; x.w -= v[4 * k + 3] + v2[4 * k + 3];
-          w4[c * 8 + k] = x;
+        for (int k = 0; k < 8; ++k) {                  // 16-byte chunk k of the row sits at chunk k ^ (row % 8)
+          float4 x;
+          x.x = -(v[4 * k] + v2[4 * k]);         x.y = -(v[4 * k + 1] + v2[4 * k + 1]);
+          x.z = -(v[4 * k + 2] + v2[4 * k + 2]); x.w = -(v[4 * k + 3] + v2[4 * k + 3]);
+          *reinterpret_cast<float4*>(my_row + ((k ^ (lane & 7)) << 4)) = x;
+        }
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          ptx::tma_reduce_add_2d(&tmW, static_cast<int>(p.c0) + t * kTileN + half * 64 + c * 32, mrow + q * 32, stage_tile);
+          ptx::bulk_commit();
         }
       }
       ptx::tc_fence_before_sync();
@@ -199,6 +208,7 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
       if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
       acc_phase[buf] ^= 1u;
     }
+    if (lane == 0) ptx::bulk_wait_all();               // every add of this warp is complete before the CTA ends
   }
 
   ptx::tc_fence_before_sync();
@@ -261,7 +271,7 @@ slice_u_kernel(const float* __restrict__ U, int64_t in, __nv_bfloat16* __restric
 // Host-side state of one GPTQ call's trailing updates: the six tensor maps never change
 // between blocks, only the coordinates do.
 struct TrailPlan {
-  CUtensorMap e[3], u[3];
+  CUtensorMap e[3], u[3], w;
   float* Wc;
   int64_t rows_total, in;
   int sm_count;
@@ -283,6 +293,11 @@ int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const
     if (rc != ADADIM_OK) return rc;
     rc = make_tmap_bf16(&plan->u[k], u[k], static_cast<uint64_t>(in), static_cast<uint64_t>(in),
                         static_cast<uint64_t>(in) * 2, 32);
+    if (rc != ADADIM_OK) return rc;
+  }
+  {
+    int rc = make_tmap_f32(&plan->w, Wc, static_cast<uint64_t>(in), static_cast<uint64_t>(rows_total),
+                           static_cast<uint64_t>(in) * 4, 32);
     if (rc != ADADIM_OK) return rc;
   }
   int dev = 0;
@@ -310,7 +325,7 @@ int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_
   if (nsplit < 1) nsplit = 1;
   if (nsplit > p.ntiles) nsplit = p.ntiles;
   trail_kernel<<<dim3(nsplit, mblocks), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],
-                                                                      plan.u[1], plan.u[2], p);
+                                                                      plan.u[1], plan.u[2], plan.w, p);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 
