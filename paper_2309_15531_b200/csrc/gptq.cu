@@ -200,13 +200,23 @@ block_kernel(const BlockArgs a) {
   const int64_t row = row0 + tid;
   float* Wd = a.Wc + static_cast<int64_t>(d) * a.out * a.in;
 
-  // stage the slab and the U block (coalesced), then work row-per-thread
-  for (int e = tid; e < kBlk * kBlk / 4; e += kBlk) {
-    int r = e >> 5, c4 = (e & 31) * 4;
-    float4 w = *reinterpret_cast<const float4*>(Wd + (row0 + r) * a.in + a.i1 + c4);
-    Ws[r * kPad + c4 + 0] = w.x; Ws[r * kPad + c4 + 1] = w.y; Ws[r * kPad + c4 + 2] = w.z; Ws[r * kPad + c4 + 3] = w.w;
-    *reinterpret_cast<float4*>(Us + r * kBlk + c4) =
-        *reinterpret_cast<const float4*>(a.U + static_cast<int64_t>(a.i1 + r) * a.in + a.i1 + c4);
+  // stage the slab and the U block (coalesced), then work row-per-thread; eight rows' worth of
+  // loads are in flight before the first is stored, so the copy costs 4 memory latencies, not 32
+#pragma unroll 1
+  for (int e0 = 0; e0 < kBlk * kBlk / 4; e0 += 8 * kBlk) {
+    float4 wv[8], uv[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
+      wv[u] = *reinterpret_cast<const float4*>(Wd + (row0 + r) * a.in + a.i1 + c4);
+      uv[u] = *reinterpret_cast<const float4*>(a.U + static_cast<int64_t>(a.i1 + r) * a.in + a.i1 + c4);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
+      Ws[r * kPad + c4 + 0] = wv[u].x; Ws[r * kPad + c4 + 1] = wv[u].y; Ws[r * kPad + c4 + 2] = wv[u].z; Ws[r * kPad + c4 + 3] = wv[u].w;
+      *reinterpret_cast<float4*>(Us + r * kBlk + c4) = uv[u];
+    }
   }
   __syncthreads();
   invd[tid] = 1.0f / Us[tid * kBlk + tid];
@@ -329,18 +339,21 @@ block_kernel(const BlockArgs a) {
   }
   __syncthreads();
   const int64_t ebase = (static_cast<int64_t>(d) * a.out + row0) * kBlk;
-  for (int e = tid; e < kBlk * kBlk; e += kBlk) {
-    const int r = e >> 7;
-    const float v = Es[r * kPad + (e & 127)];
-    const float g = invd[r], inv = 1.0f / g;        // powers of two: exact
+  // thread tid takes column tid of every row r (e = 128 r + tid): a warp stores 64 contiguous bytes
+#pragma unroll 8
+  for (int r = 0; r < kBlk; ++r) {
+    const float v = Es[r * kPad + tid];
+    const float g = invd[r];
+    const float inv = __int_as_float(0x7F000000 - __float_as_int(g));   // 1 / g for a power of two, exact
     const float a0 = rintf(v * inv);
     const float r1 = fmaf(-a0, g, v);
     const float a1 = rintf(r1 * inv * 256.0f);
     const float r2 = fmaf(-a1, g * (1.0f / 256.0f), r1);
     const float a2 = rintf(r2 * inv * 65536.0f);
-    a.Ep[0][ebase + e] = __float2bfloat16_rn(a0 * g);
-    a.Ep[1][ebase + e] = __float2bfloat16_rn(a1 * g * (1.0f / 256.0f));
-    a.Ep[2][ebase + e] = __float2bfloat16_rn(a2 * g * (1.0f / 65536.0f));
+    const int64_t e = ebase + static_cast<int64_t>(r) * kBlk + tid;
+    a.Ep[0][e] = __float2bfloat16_rn(a0 * g);
+    a.Ep[1][e] = __float2bfloat16_rn(a1 * g * (1.0f / 256.0f));
+    a.Ep[2][e] = __float2bfloat16_rn(a2 * g * (1.0f / 65536.0f));
   }
   if (is_ic) {
     for (int e = tid; e < NG * kBlk; e += kBlk) {
