@@ -177,6 +177,42 @@ __device__ __forceinline__ int ordered_key(float v) {
 }
 __device__ __forceinline__ float from_ordered_key(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7fffffff)); }
 
+// W[:, later columns] -= Err[:, this sub-block] * U[sub-block rows, later columns] for the whole
+// 128-row slab in shared memory.  A row-per-thread loop needs one warp-uniform U value per
+// multiply-add, all of it through the shared-memory return path, which bounds it at a quarter of
+// the multiply-add rate; here a thread owns 8 rows x CW columns, so 8 + CW loads feed 8 CW
+// multiply-adds.  Every element still receives its 32 updates in the same order as before.
+template <int CW>
+__device__ __forceinline__ void lazy_update(float* __restrict__ Ws, const float* __restrict__ Us,
+                                            const float* __restrict__ Es, int cbase, int tid) {
+  const int r0 = (tid >> 3) * 8;
+  const int col0 = cbase + kSub + (tid & 7) * CW;
+  float acc[8][CW];
+#pragma unroll
+  for (int m = 0; m < 8; ++m)
+#pragma unroll
+    for (int n = 0; n < CW; ++n) acc[m][n] = Ws[(r0 + m) * kPad + col0 + n];
+#pragma unroll 4
+  for (int ii = 0; ii < kSub; ++ii) {
+    float e[8], u[CW];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) e[m] = Es[(r0 + m) * kPad + cbase + ii];
+#pragma unroll
+    for (int n4 = 0; n4 < CW / 4; ++n4) {
+      const float4 t = *reinterpret_cast<const float4*>(Us + (cbase + ii) * kBlk + col0 + 4 * n4);
+      u[4 * n4] = t.x; u[4 * n4 + 1] = t.y; u[4 * n4 + 2] = t.z; u[4 * n4 + 3] = t.w;
+    }
+#pragma unroll
+    for (int m = 0; m < 8; ++m)
+#pragma unroll
+      for (int n = 0; n < CW; ++n) acc[m][n] = fmaf(-e[m], u[n], acc[m][n]);
+  }
+#pragma unroll
+  for (int m = 0; m < 8; ++m)
+#pragma unroll
+    for (int n = 0; n < CW; ++n) Ws[(r0 + m) * kPad + col0 + n] = acc[m][n];
+}
+
 template <int BITS, int G>
 __global__ void __launch_bounds__(kBlk, 1)
 block_kernel(const BlockArgs a) {
@@ -304,27 +340,14 @@ block_kernel(const BlockArgs a) {
     uint32_t* cdst = a.codes[d] + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
 #pragma unroll
     for (int k = 0; k < BITS; ++k) cdst[k] = cw[k];
-    // lazy update of the block's later columns with this sub-block's 32 errors
-#pragma unroll 1
-    for (int jc = cbase + kSub; jc < kBlk; jc += kSub) {
-      float acc[kSub];
-#pragma unroll
-      for (int k = 0; k < kSub; ++k) acc[k] = wrow[jc + k];
-#pragma unroll
-      for (int ii = 0; ii < kSub; ++ii) {
-        const float4* u4 = reinterpret_cast<const float4*>(Us + (cbase + ii) * kBlk + jc);
-#pragma unroll
-        for (int k4 = 0; k4 < kSub / 4; ++k4) {
-          float4 u = u4[k4];
-          acc[k4 * 4 + 0] = fmaf(-err[ii], u.x, acc[k4 * 4 + 0]);
-          acc[k4 * 4 + 1] = fmaf(-err[ii], u.y, acc[k4 * 4 + 1]);
-          acc[k4 * 4 + 2] = fmaf(-err[ii], u.z, acc[k4 * 4 + 2]);
-          acc[k4 * 4 + 3] = fmaf(-err[ii], u.w, acc[k4 * 4 + 3]);
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < kSub; ++k) wrow[jc + k] = acc[k];
-    }
+    // lazy update of the block's later columns with this sub-block's 32 errors, as a small
+    // register-tiled product over the whole slab (see lazy_update)
+    __syncthreads();
+    const int later = kBlk - cbase - kSub;
+    if (later == 96) lazy_update<12>(Ws, Us, Es, cbase, tid);
+    else if (later == 64) lazy_update<8>(Ws, Us, Es, cbase, tid);
+    else if (later == 32) lazy_update<4>(Ws, Us, Es, cbase, tid);
+    __syncthreads();
   }
 
   // ---- outputs: errors (coalesced), per-IC parameters, loss ------------------------------
