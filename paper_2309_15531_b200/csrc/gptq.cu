@@ -25,7 +25,7 @@ struct TrailPlan {
 int trail_split_u(const float* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st);
 int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
                const __nv_bfloat16* const u[3]);
-int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_ctas, int* status_dev, cudaStream_t st);
+int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int tiles_per_cta, int* status_dev, cudaStream_t st);
 
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
@@ -519,7 +519,7 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   if (rc0 != ADADIM_OK) return rc0;
   // Block b+1 only needs its own 128 columns from block b's trailing update.  That part runs on a
   // high-priority stream together with the block kernels; the rest of each trailing update runs
-  // beside the next block kernel on a second stream, on few enough CTAs to leave it room.  The
+  // beside the next block kernel on a second stream, on the SMs the block kernel leaves free.  The
   // error pieces alternate between two sets, so a block kernel never overwrites what the other
   // stream still reads.
   cudaStream_t chain = nullptr, side = nullptr;
@@ -535,8 +535,11 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   ADADIM_CUDA_TRY(cudaEventRecord(ev_fork, st));
   ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_fork, 0));
   const int64_t rows_total = static_cast<int64_t>(ndim) * out;
-  const int block_ctas = slabs * ndim;
-  const int rest_ctas = plan.sm_count - block_ctas > 0 ? plan.sm_count - block_ctas : 1;
+  // the side-stream launches get the SMs that the block kernel leaves free (finer CTAs were
+  // measured slower: every CTA reloads its 96 KB of error pieces and refills the pipeline)
+  const int free_sms = plan.sm_count - slabs * ndim;
+  const int64_t mblocks = rows_total / kBlk;
+  const int rest_split = free_sms >= mblocks ? static_cast<int>(free_sms / mblocks) : 1;
   __nv_bfloat16* ep_base[3] = {a.Ep[0], a.Ep[1], a.Ep[2]};
   bool rest_pending = false;
   for (int i1 = 0; i1 < in; i1 += kBlk) {
@@ -557,11 +560,12 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
       // the next block's columns were last written by the previous block's side-stream launch
       if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
       rest_pending = false;
-      rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, plan.sm_count, status_dev, chain);
+      rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, 1, status_dev, chain);
       if (rc != ADADIM_OK) return rc;
       if (tiles_after > 1) {
         ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_block, 0));
-        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1, rest_ctas, status_dev, side);
+        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1,
+                          (tiles_after - 1 + rest_split - 1) / rest_split, status_dev, side);
         if (rc != ADADIM_OK) return rc;
         ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
         rest_pending = true;

@@ -309,8 +309,10 @@ int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const
 }
 
 // Updates `ntiles` 128-column tiles starting at column c0 with the errors of the block whose first
-// column is i1 (error set i1/128 & 1), on at most max_ctas CTAs.
-int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_ctas, int* status_dev, cudaStream_t st) {
+// column is i1 (error set i1/128 & 1); every CTA takes about `tiles_per_cta` tiles of one 128-row
+// block.  Small CTAs let a launch that runs beside higher-priority kernels use whatever SMs are
+// idle and hand them back quickly.
+int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int tiles_per_cta, int* status_dev, cudaStream_t st) {
   TrailParams p;
   p.Wc = plan.Wc;
   p.in = plan.in;
@@ -321,9 +323,8 @@ int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_
   p.status_dev = status_dev;
   if (p.ntiles <= 0) return ADADIM_OK;
   const int mblocks = static_cast<int>(plan.rows_total / 128);
-  int nsplit = max_ctas / mblocks;
+  int nsplit = (ntiles + tiles_per_cta - 1) / tiles_per_cta;
   if (nsplit < 1) nsplit = 1;
-  if (nsplit > p.ntiles) nsplit = p.ntiles;
   trail_kernel<<<dim3(nsplit, mblocks), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],
                                                                       plan.u[1], plan.u[2], plan.w, p);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;

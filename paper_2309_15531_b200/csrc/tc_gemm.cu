@@ -86,6 +86,7 @@ struct TcParams {
 constexpr int kKT = 64;                       // reduction depth of one ring stage
 constexpr int kTcThreads = 192;
 constexpr uint32_t kOperandBytes = 256 * kKT * 2;   // one 256-wide bf16 operand slab per stage
+constexpr uint32_t kOutChunk = 32 * 32 * 4;          // one epilogue warp's staging tile: 32 rows x 32 fp32 columns
 
 template <Mode MODE> struct TcCfg;
 template <> struct TcCfg<Mode::kHessian> { static constexpr int NB = 1, STAGES = 3; static constexpr bool MN = true; };
@@ -93,7 +94,7 @@ template <> struct TcCfg<Mode::kGram>    { static constexpr int NB = 1, STAGES =
 
 template <Mode MODE>
 constexpr size_t tc_smem_bytes() {
-  return static_cast<size_t>(TcCfg<MODE>::STAGES) * (1 + TcCfg<MODE>::NB) * kOperandBytes + 1024 + 256;
+  return static_cast<size_t>(TcCfg<MODE>::STAGES) * (1 + TcCfg<MODE>::NB) * kOperandBytes + 4 * kOutChunk + 1024 + 256;
 }
 
 __device__ __forceinline__ void tri_coords(int t, int& rb, int& cb) {
@@ -114,7 +115,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint8_t* out_smem = smem + STAGES * STAGE_BYTES;     // [4 warps][32 rows][128 B], 128-byte swizzle (Hessian drains)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 4 * kOutChunk);
   uint64_t* full = bars;                   // [STAGES] TMA -> MMA
   uint64_t* empty = bars + STAGES;         // [STAGES] MMA -> TMA
   uint64_t* acc_full = bars + 2 * STAGES;  // MMA -> epilogue
@@ -241,6 +243,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;                       // TMEM lane quadrant this warp may read
     uint32_t acc_phase = 0;
+    uint8_t* stage_tile = out_smem + q * kOutChunk;
+    uint8_t* my_row = stage_tile + lane * 128;    // this lane's row of the staging tile
     for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
       int rb, cb;
       tri_coords(MODE == Mode::kGram ? t % p.tiles_per_dim : t, rb, cb);
@@ -249,6 +253,12 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       live = ptx::mbar_wait(acc_full, acc_phase, dead, p.status_dev);
       if (!live) break;
       ptx::tc_fence_after_sync();
+      // The adds of the previous drain went to the same elements of H: they must be complete
+      // before this drain's are issued, or the order of the two roundings would not be fixed.
+      if (MODE == Mode::kHessian) {
+        if (lane == 0) ptx::bulk_wait_all();
+        __syncwarp();
+      }
       double part[2] = {0.0, 0.0};
 #pragma unroll 1
       for (int a = 0; a < 2; ++a) {
@@ -259,16 +269,25 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           ptx::tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * 256 + c * 32, v);
           const int64_t j0 = static_cast<int64_t>(cb) * 256 + c * 32;
           if (MODE == Mode::kHessian) {
-            if (i < p.in) {
-              float* hrow = p.H + i * p.in + j0;
+            // H += 2 acc as an element-wise add done by the memory system: the doubled values go
+            // to a swizzled staging tile and from there into H, 32 rows x 32 columns at a time
+            // (the part of a tile outside the matrix is not written).  H is never read here.
+            const int64_t i0 = static_cast<int64_t>(rb) * 256 + a * 128 + q * 32;
+            if (i0 < p.in && j0 < p.in) {
+              if (lane == 0) ptx::bulk_wait_read();   // the previous add has finished reading the staging tile
+              __syncwarp();
 #pragma unroll
-              for (int k4 = 0; k4 < 8; ++k4) {
-                if (j0 + k4 * 4 < p.in) {
-                  float4 h = *reinterpret_cast<float4*>(hrow + k4 * 4);
-                  h.x += 2.0f * v[k4 * 4 + 0]; h.y += 2.0f * v[k4 * 4 + 1];
-                  h.z += 2.0f * v[k4 * 4 + 2]; h.w += 2.0f * v[k4 * 4 + 3];
-                  *reinterpret_cast<float4*>(hrow + k4 * 4) = h;
-                }
+              for (int k4 = 0; k4 < 8; ++k4) {        // 16-byte chunk k4 of the row sits at chunk k4 ^ (row % 8)
+                float4 x;
+                x.x = 2.0f * v[k4 * 4 + 0]; x.y = 2.0f * v[k4 * 4 + 1];
+                x.z = 2.0f * v[k4 * 4 + 2]; x.w = 2.0f * v[k4 * 4 + 3];
+                *reinterpret_cast<float4*>(my_row + ((k4 ^ (lane & 7)) << 4)) = x;
+              }
+              ptx::fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                ptx::tma_reduce_add_2d(&tmB1, static_cast<int>(j0), static_cast<int>(i0), stage_tile);
+                ptx::bulk_commit();
               }
             }
           } else {
@@ -306,6 +325,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       }
       if (!live) break;
     }
+    if (MODE == Mode::kHessian && lane == 0) ptx::bulk_wait_all();   // every add is complete before the CTA ends
   }
 
   ptx::tc_fence_before_sync();
@@ -416,7 +436,10 @@ int hessian_bf16_launch(const void* X, int64_t n_tokens, int64_t in, int64_t ldx
   p.status_dev = status_dev;
   p.H = H;
   p.in = in;
-  rc = tc_launch<Mode::kHessian>(tm, tm, tm, p, st);
+  CUtensorMap th;                                      // H itself, for the element-wise adds of the drains
+  rc = make_tmap_f32(&th, H, static_cast<uint64_t>(in), static_cast<uint64_t>(in), static_cast<uint64_t>(in) * 4, 32);
+  if (rc != ADADIM_OK) return rc;
+  rc = tc_launch<Mode::kHessian>(tm, tm, th, p, st);
   if (rc != ADADIM_OK) return rc;
   const unsigned nt = static_cast<unsigned>((in + 31) / 32);
   if (nblk > 1) mirror_kernel<<<dim3(nt, nt), 256, 0, st>>>(H, in);
