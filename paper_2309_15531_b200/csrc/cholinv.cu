@@ -28,55 +28,78 @@ constexpr int kGroup = 4;   // panels per rank-256 update
 
 __host__ __device__ __forceinline__ int64_t mn64(int64_t a, int64_t b) { return a < b ? a : b; }
 
-// ---- 64 x 64 output tile product, 256 threads, 4 x 4 outputs per thread --------------------
+// D += A B on 8 x 8 x 4 fp64 fragments: lane l holds A[l/4][l%4], B[l%4][l/4] and the two
+// outputs D[l/4][2 (l%4)], D[l/4][2 (l%4) + 1].
+__device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
+}
+
+// ---- 64 x 64 output tile product (K = 64) on the fp64 matrix instruction, 256 threads ---------
 // acc += A[64 x 64] * B, A row-major with leading dimension lda;
 // B_T: B is given as [64 cols][64] row-major (product with the transpose), else as [64][64 cols].
-// These tiles sit on the factorization's critical chain, so every global load of the tile is
-// issued before the first one is used: one memory latency per tile instead of one per slab.
+// Each of the eight warps owns 32 rows x 16 columns as 4 x 2 fragments.  These tiles sit on the
+// factorization's critical chain, so every global load of both operands is issued before the
+// first one is used (one memory latency per tile), and the operands are staged in two K-halves.
+// The row pitch is 8 mod 16 doubles: a fragment's 4 k-rows x 8 columns fall on distinct banks.
+constexpr int kHalfK = kNB / 2;
+#define TILE_SMEM                           \
+  __shared__ double sa[kHalfK][kNB + 8];    \
+  __shared__ double sb[kHalfK][kNB + 8];
+
 template <bool B_T>
 __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64_t lda, const double* __restrict__ B,
-                                             int64_t ldb, int K, double (&acc)[4][4], double (*sa)[kNB + 2],
-                                             double (*sb)[kNB + 2]) {
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  constexpr int kSlabs = kNB / 16;
-  double2 av[kSlabs][2], bv[kSlabs][2];
-  const int r = threadIdx.x >> 2, kq = (threadIdx.x & 3) * 4;          // loader: row (or column of B^T), first k of four
-  const int kk = threadIdx.x >> 4, nq = (threadIdx.x & 15) * 4;        // loader of a non-transposed B: k row, first column
+                                             int64_t ldb, double (&acc)[4][2][2], double (*sa)[kNB + 8],
+                                             double (*sb)[kNB + 8]) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 1) * 32, wn = (warp >> 1) * 16;
+  const int fk = lane & 3, fr = lane >> 2;
+  const int r = tid >> 2, kq = (tid & 3) * 8;            // loader: row (or column of B^T), first k of eight
+  const int kk = tid >> 3, nq = (tid & 7) * 8;           // loader of a non-transposed B: k row, first column of eight
+  double2 av[2][4], bv[2][4];
 #pragma unroll
-  for (int sl = 0; sl < kSlabs; ++sl) {
-    const double2* asrc = reinterpret_cast<const double2*>(A + static_cast<int64_t>(r) * lda + sl * 16 + kq);
-    av[sl][0] = asrc[0]; av[sl][1] = asrc[1];
-    const double2* bsrc = B_T ? reinterpret_cast<const double2*>(B + static_cast<int64_t>(r) * ldb + sl * 16 + kq)
-                              : reinterpret_cast<const double2*>(B + static_cast<int64_t>(sl * 16 + kk) * ldb + nq);
-    bv[sl][0] = bsrc[0]; bv[sl][1] = bsrc[1];
+  for (int h = 0; h < 2; ++h) {
+    const double2* asrc = reinterpret_cast<const double2*>(A + static_cast<int64_t>(r) * lda + h * kHalfK + kq);
+    const double2* bsrc = B_T ? reinterpret_cast<const double2*>(B + static_cast<int64_t>(r) * ldb + h * kHalfK + kq)
+                              : reinterpret_cast<const double2*>(B + static_cast<int64_t>(h * kHalfK + kk) * ldb + nq);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { av[h][t] = asrc[t]; bv[h][t] = bsrc[t]; }
   }
-  (void)K;
 #pragma unroll
-  for (int sl = 0; sl < kSlabs; ++sl) {
-    sa[kq + 0][r] = av[sl][0].x; sa[kq + 1][r] = av[sl][0].y; sa[kq + 2][r] = av[sl][1].x; sa[kq + 3][r] = av[sl][1].y;
-    if (B_T) {
-      sb[kq + 0][r] = bv[sl][0].x; sb[kq + 1][r] = bv[sl][0].y; sb[kq + 2][r] = bv[sl][1].x; sb[kq + 3][r] = bv[sl][1].y;
-    } else {
-      sb[kk][nq + 0] = bv[sl][0].x; sb[kk][nq + 1] = bv[sl][0].y; sb[kk][nq + 2] = bv[sl][1].x; sb[kk][nq + 3] = bv[sl][1].y;
+  for (int h = 0; h < 2; ++h) {
+    if (h > 0) __syncthreads();                          // the first half has been consumed
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      sa[kq + 2 * t][r] = av[h][t].x; sa[kq + 2 * t + 1][r] = av[h][t].y;
+      if (B_T) { sb[kq + 2 * t][r] = bv[h][t].x; sb[kq + 2 * t + 1][r] = bv[h][t].y; }
+      else *reinterpret_cast<double2*>(&sb[kk][nq + 2 * t]) = bv[h][t];
     }
     __syncthreads();
 #pragma unroll
-    for (int k2 = 0; k2 < 16; ++k2) {
-      double a[4], b[4];
+    for (int ks = 0; ks < kHalfK; ks += 4) {
+      double af[4], bf[2];
 #pragma unroll
-      for (int m = 0; m < 4; ++m) { a[m] = sa[k2][ty * 4 + m]; b[m] = sb[k2][tx * 4 + m]; }
+      for (int i = 0; i < 4; ++i) af[i] = sa[ks + fk][wm + 8 * i + fr];
 #pragma unroll
-      for (int m = 0; m < 4; ++m)
+      for (int j = 0; j < 2; ++j) bf[j] = sb[ks + fk][wn + 8 * j + fr];
 #pragma unroll
-        for (int n = 0; n < 4; ++n) acc[m][n] = fma(a[m], b[n], acc[m][n]);
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) mma_f64(acc[i][j], af[i], bf[j]);
     }
-    __syncthreads();
   }
 }
 
-#define TILE_SMEM                      \
-  __shared__ double sa[16][kNB + 2];   \
-  __shared__ double sb[16][kNB + 2];
+// Applies f(row, first column, values of 2 consecutive columns) to a thread's outputs of the tile.
+template <typename F>
+__device__ __forceinline__ void for_each_pair64(double (&acc)[4][2][2], F f) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int wm = (warp & 1) * 32, wn = (warp >> 1) * 16;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) f(wm + 8 * i + (lane >> 2), wn + 8 * j + 2 * (lane & 3), acc[i][j]);
+}
 
 // ---- 128 x 64 output tile product on the fp64 tensor-core path, 256 threads ----------------
 // Each of the eight warps owns a 32 x 32 piece of the tile as 4 x 4 fragments of the 8 x 8 x 4
@@ -92,11 +115,6 @@ struct TileSmem {
   double a[2][kBK][kT + 8];
   double b[2][kBK][kTN + 8];
 };
-
-__device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
-  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-               : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
-}
 
 // acc[i][j] is the fragment at rows 8 i, columns 8 j of the warp's piece: this lane holds row
 // lane / 4 and columns 2 (lane % 4), 2 (lane % 4) + 1 of it.
@@ -414,13 +432,11 @@ panel_kernel(double* __restrict__ A, int64_t n, int k, const double* __restrict_
   TILE_SMEM
   const int64_t row0 = (static_cast<int64_t>(k) + 1 + blockIdx.x) * kNB;
   double* tile = A + row0 * n + static_cast<int64_t>(k) * kNB;
-  double acc[4][4] = {};
-  tile_product<true>(tile, n, dinv + static_cast<int64_t>(k) * kNB * kNB, kNB, kNB, acc, sa, sb);
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-#pragma unroll
-  for (int m = 0; m < 4; ++m)
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tile[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + c] = acc[m][c];
+  double acc[4][2][2] = {};
+  tile_product<true>(tile, n, dinv + static_cast<int64_t>(k) * kNB * kNB, kNB, acc, sa, sb);
+  for_each_pair64(acc, [&](int r, int c, const double* v) {
+    *reinterpret_cast<double2*>(tile + static_cast<int64_t>(r) * n + c) = make_double2(v[0], v[1]);
+  });
 }
 
 // Update inside the current group of panels after panel k:  A[i][j] -= L[i][k] L[j][k]^T for the
@@ -432,14 +448,15 @@ group_update_kernel(double* __restrict__ A, int64_t n, int k) {
   if (blockIdx.y > blockIdx.x) return;
   const int64_t ri = (static_cast<int64_t>(k) + 1 + blockIdx.x) * kNB, rj = (static_cast<int64_t>(k) + 1 + blockIdx.y) * kNB;
   const int64_t ck = static_cast<int64_t>(k) * kNB;
-  double acc[4][4] = {};
-  tile_product<true>(A + ri * n + ck, n, A + rj * n + ck, n, kNB, acc, sa, sb);
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  double* c = A + ri * n + rj;
-#pragma unroll
-  for (int m = 0; m < 4; ++m)
-#pragma unroll
-    for (int q = 0; q < 4; ++q) c[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + q] -= acc[m][q];
+  double acc[4][2][2] = {};
+  tile_product<true>(A + ri * n + ck, n, A + rj * n + ck, n, acc, sa, sb);
+  double* c0 = A + ri * n + rj;
+  for_each_pair64(acc, [&](int r, int c, const double* v) {
+    double2* p = reinterpret_cast<double2*>(c0 + static_cast<int64_t>(r) * n + c);
+    double2 u = *p;
+    u.x -= v[0]; u.y -= v[1];
+    *p = u;
+  });
 }
 
 // Rank-`kw` update of everything right of a finished group:  for tiles of 128 rows x 64 columns on
@@ -502,28 +519,24 @@ merge1_64_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ T
   TILE_SMEM
   const int64_t s = kNB, a0 = static_cast<int64_t>(blockIdx.x) * 2 * s, b0 = a0 + s;
   if (b0 >= n) return;
-  double acc[4][4] = {};
-  tile_product<false>(A + b0 * n + a0, n, A + a0 * n + a0, n, kNB, acc, sa, sb);
+  double acc[4][2][2] = {};
+  tile_product<false>(A + b0 * n + a0, n, A + a0 * n + a0, n, acc, sa, sb);
   double* t = T + static_cast<int64_t>(blockIdx.x) * s * s;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-#pragma unroll
-  for (int m = 0; m < 4; ++m)
-#pragma unroll
-    for (int q = 0; q < 4; ++q) t[(ty * 4 + m) * s + tx * 4 + q] = acc[m][q];
+  for_each_pair64(acc, [&](int r, int c, const double* v) {
+    *reinterpret_cast<double2*>(t + r * s + c) = make_double2(v[0], v[1]);
+  });
 }
 __global__ void __launch_bounds__(256)
 merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T) {      // s == 64
   TILE_SMEM
   const int64_t s = kNB, a0 = static_cast<int64_t>(blockIdx.x) * 2 * s, b0 = a0 + s;
   if (b0 >= n) return;
-  double acc[4][4] = {};
-  tile_product<false>(A + b0 * n + b0, n, T + static_cast<int64_t>(blockIdx.x) * s * s, s, kNB, acc, sa, sb);
+  double acc[4][2][2] = {};
+  tile_product<false>(A + b0 * n + b0, n, T + static_cast<int64_t>(blockIdx.x) * s * s, s, acc, sa, sb);
   double* dst = A + b0 * n + a0;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-#pragma unroll
-  for (int m = 0; m < 4; ++m)
-#pragma unroll
-    for (int q = 0; q < 4; ++q) dst[static_cast<int64_t>(ty * 4 + m) * n + tx * 4 + q] = -acc[m][q];
+  for_each_pair64(acc, [&](int r, int c, const double* v) {
+    *reinterpret_cast<double2*>(dst + static_cast<int64_t>(r) * n + c) = make_double2(-v[0], -v[1]);
+  });
 }
 
 __global__ void __launch_bounds__(256, 2)
