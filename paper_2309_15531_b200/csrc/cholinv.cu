@@ -195,6 +195,73 @@ __device__ __forceinline__ void for_each_pair(double (&acc)[4][4][2], F f) {
     for (int j = 0; j < 4; ++j) f(wm + 8 * i + (lane >> 2), wn + 8 * j + 2 * (lane & 3), acc[i][j]);
 }
 
+// ---- 64 x 64 output tile product with any K (a multiple of 8), same scheme as the 128 x 64 one --
+// Used where a launch has few tiles or long reductions (the rank update of the next group's own
+// columns; the merges, whose longest reductions decide the kernel's length): half the work per
+// CTA, twice the CTAs.  Warps own 32 x 16 pieces (4 x 2 fragments) as in tile_product.
+struct TileSmem64 {
+  double a[2][kBK][kNB + 8];
+  double b[2][kBK][kNB + 8];
+};
+
+template <bool B_T>
+__device__ __forceinline__ void product_tile64(const double* __restrict__ A, int64_t lda,
+                                               const double* __restrict__ B, int64_t ldb, int K,
+                                               double (&acc)[4][2][2], TileSmem64& sm) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 1) * 32, wn = (warp >> 1) * 16;
+  const int fk = lane & 3, fr = lane >> 2;
+  const int ar = tid >> 2, akq = (tid & 3) * 2;                 // A / B^T loader: row, first k of two
+  const int bkk = tid >> 5, bnq = (tid & 31) * 2;               // B loader (not transposed): k row, first col of two
+  const double* ap = A + static_cast<int64_t>(ar) * lda + akq;
+  const double* bp = B_T ? B + static_cast<int64_t>(ar) * ldb + akq : B + static_cast<int64_t>(bkk) * ldb + bnq;
+  const int64_t bstep = B_T ? kBK : static_cast<int64_t>(kBK) * ldb;
+  struct Slab { double2 a, b; };
+  Slab s0, s1;
+
+  auto fetch = [&](Slab& r, int k0) {
+    r.a = *reinterpret_cast<const double2*>(ap + k0);
+    r.b = *reinterpret_cast<const double2*>(bp + (k0 / kBK) * bstep);
+  };
+  auto stash = [&](const Slab& r, int buf) {
+    sm.a[buf][akq][ar] = r.a.x; sm.a[buf][akq + 1][ar] = r.a.y;
+    if (B_T) { sm.b[buf][akq][ar] = r.b.x; sm.b[buf][akq + 1][ar] = r.b.y; }
+    else *reinterpret_cast<double2*>(&sm.b[buf][bkk][bnq]) = r.b;
+  };
+  auto multiply = [&](int buf) {
+#pragma unroll
+    for (int ks = 0; ks < kBK; ks += 4) {
+      double af[4], bf[2];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) af[i] = sm.a[buf][ks + fk][wm + 8 * i + fr];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) bf[j] = sm.b[buf][ks + fk][wn + 8 * j + fr];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) mma_f64(acc[i][j], af[i], bf[j]);
+    }
+  };
+
+  const int nslab = K / kBK;
+  fetch(s0, 0);
+  if (nslab > 1) fetch(s1, kBK);
+  stash(s0, 0);
+  __syncthreads();
+  for (int i = 0; i < nslab; i += 2) {
+    if (i + 1 < nslab) stash(s1, 1);
+    if (i + 2 < nslab) fetch(s0, (i + 2) * kBK);
+    multiply(0);
+    __syncthreads();
+    if (i + 1 < nslab) {
+      if (i + 2 < nslab) stash(s0, 0);
+      if (i + 3 < nslab) fetch(s1, (i + 3) * kBK);
+      multiply(1);
+      __syncthreads();
+    }
+  }
+}
+
 // ---- set-up --------------------------------------------------------------------------------
 // stats[0] = lambda = percdamp * mean_i diag(H) after the dead-column fix (fixed summation order).
 __global__ void __launch_bounds__(256)
@@ -459,31 +526,41 @@ group_update_kernel(double* __restrict__ A, int64_t n, int k) {
   });
 }
 
-// Rank-`kw` update of everything right of a finished group:  for tiles of 128 rows x 64 columns on
-// or below the diagonal of the region starting at row/column e:
-//   A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T.
-// Row block ti meets column blocks 0 .. 2*ti+1.  The tile right of the diagonal 64-block (column
-// block 2*ti+1) only stores its lower 64 rows: the block above them must stay zero.
+// Rank-`kw` update of everything right of a finished group, for the region starting at row/column e:
+//   A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T   on and below the diagonal.
 // The update is issued in two parts so that the next group's factorization can start early:
-// `first_cols` launches a (kLook, row blocks) grid over the first kLook column blocks (the next
-// group's own columns); the other launch walks the whole triangle and skips those.
+//  * the next group's own columns [e, e + 256): rank_update_first_kernel, 64 x 64 tiles, one wave
+//    of short CTAs on the high-priority chain;
+//  * the rest: rank_update_kernel, 128 x 64 tiles over the whole triangle, skipping those columns.
+// In the second kernel row block ti meets column blocks 0 .. 2*ti+1; the tile right of the diagonal
+// 64-block (column block 2*ti+1) only stores its lower 64 rows: the block above them must stay zero.
 constexpr int kLook = kGroup * kNB / kTN;
 __global__ void __launch_bounds__(256, 2)
-rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw, bool first_cols) {
+rank_update_first_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
+  __shared__ TileSmem64 sm;
+  const int ti = blockIdx.y, cj = blockIdx.x;               // 64-row block, 64-column block of the region
+  if (cj > ti) return;
+  const int64_t ri = e + static_cast<int64_t>(ti) * kNB, rj = e + static_cast<int64_t>(cj) * kNB;
+  if (rj >= n) return;
+  double acc[4][2][2] = {};
+  product_tile64<true>(A + ri * n + j0, n, A + rj * n + j0, n, kw, acc, sm);
+  for_each_pair64(acc, [&](int r, int c2, const double* v) {
+    double2* p = reinterpret_cast<double2*>(A + (ri + r) * n + rj + c2);
+    double2 u = *p;
+    u.x -= v[0]; u.y -= v[1];
+    *p = u;
+  });
+}
+
+__global__ void __launch_bounds__(256, 2)
+rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
   __shared__ TileSmem sm;
-  int ti, cj;
-  if (first_cols) {
-    ti = blockIdx.y;
-    cj = blockIdx.x;
-    if (cj > 2 * ti + 1) return;
-  } else {
-    const int t = blockIdx.x;
-    ti = static_cast<int>((sqrt(4.0 * t + 1.0) - 1.0) * 0.5);
-    while (ti * (ti + 1) > t) --ti;
-    while ((ti + 1) * (ti + 2) <= t) ++ti;
-    cj = t - ti * (ti + 1);
-    if (cj < kLook) return;
-  }
+  const int t = blockIdx.x;
+  int ti = static_cast<int>((sqrt(4.0 * t + 1.0) - 1.0) * 0.5);
+  while (ti * (ti + 1) > t) --ti;
+  while ((ti + 1) * (ti + 2) <= t) ++ti;
+  const int cj = t - ti * (ti + 1);
+  if (cj < kLook) return;
   const int64_t ri = e + static_cast<int64_t>(ti) * kT, rj = e + static_cast<int64_t>(cj) * kTN;
   if (rj >= n) return;
   const int vr = static_cast<int>(mn64(kT, n - ri));
@@ -541,44 +618,40 @@ merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T
 
 __global__ void __launch_bounds__(256, 2)
 merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T) {      // s >= 128
-  __shared__ TileSmem sm;
+  __shared__ TileSmem64 sm;
   const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  // 128-row block r, 64-column block c; the reduction length s - 64 c falls with c, so tiles are
+  // 64-row block r, 64-column block c; the reduction length s - 64 c falls with c, so tiles are
   // handed out column block by column block: the longest ones start first
-  const int rtiles = static_cast<int>(s / kT);
+  const int rtiles = static_cast<int>(s / kNB);
   const int r = blockIdx.x % rtiles, c = blockIdx.x / rtiles;
   const int64_t sB = mn64(s, n - b0);
-  if (static_cast<int64_t>(r) * kT >= sB) return;
-  const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
-  const int64_t m0 = static_cast<int64_t>(c) * kTN;
-  double acc[4][4][2] = {};
-  product_tile<false>(A + (b0 + static_cast<int64_t>(r) * kT) * n + a0 + m0, n, vr, A + (a0 + m0) * n + a0 + m0, n,
-                      static_cast<int>(s - m0), acc, sm);
-  double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kT * s + m0;
-  for_each_pair(acc, [&](int rr, int c2, const double* v) {
-    if (rr >= vr) return;
+  if (static_cast<int64_t>(r) * kNB >= sB) return;
+  const int64_t m0 = static_cast<int64_t>(c) * kNB;
+  double acc[4][2][2] = {};
+  product_tile64<false>(A + (b0 + static_cast<int64_t>(r) * kNB) * n + a0 + m0, n, A + (a0 + m0) * n + a0 + m0, n,
+                        static_cast<int>(s - m0), acc, sm);
+  double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kNB * s + m0;
+  for_each_pair64(acc, [&](int rr, int c2, const double* v) {
     *reinterpret_cast<double2*>(t + static_cast<int64_t>(rr) * s + c2) = make_double2(v[0], v[1]);
   });
 }
 __global__ void __launch_bounds__(256, 2)
 merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T) {      // s >= 128
-  __shared__ TileSmem sm;
-  const int ctiles = static_cast<int>(s / kTN);
+  __shared__ TileSmem64 sm;
+  const int ctiles = static_cast<int>(s / kNB);
   const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
-  // the reduction length 128 (r + 1) grows with the row block: the last row blocks start first
-  const int rtiles = static_cast<int>(s / kT);
+  // the reduction length 64 (r + 1) grows with the row block: the last row blocks start first
+  const int rtiles = static_cast<int>(s / kNB);
   const int r = rtiles - 1 - static_cast<int>(blockIdx.x) / ctiles, c = blockIdx.x % ctiles;
   const int64_t sB = mn64(s, n - b0);
-  if (static_cast<int64_t>(r) * kT >= sB) return;
-  const int64_t row0 = b0 + static_cast<int64_t>(r) * kT;
-  const int vr = static_cast<int>(mn64(kT, sB - static_cast<int64_t>(r) * kT));
-  const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kT, sB));
-  double acc[4][4][2] = {};
-  product_tile<false>(A + row0 * n + b0, n, vr, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kTN,
-                      s, K, acc, sm);
-  double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kTN;
-  for_each_pair(acc, [&](int rr, int c2, const double* v) {
-    if (rr >= vr) return;
+  if (static_cast<int64_t>(r) * kNB >= sB) return;
+  const int64_t row0 = b0 + static_cast<int64_t>(r) * kNB;
+  const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kNB, sB));
+  double acc[4][2][2] = {};
+  product_tile64<false>(A + row0 * n + b0, n, T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(c) * kNB,
+                        s, K, acc, sm);
+  double* dst = A + row0 * n + a0 + static_cast<int64_t>(c) * kNB;
+  for_each_pair64(acc, [&](int rr, int c2, const double* v) {
     *reinterpret_cast<double2*>(dst + static_cast<int64_t>(rr) * n + c2) = make_double2(-v[0], -v[1]);
   });
 }
@@ -657,11 +730,11 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
       if (has_rest) ADADIM_CUDA_TRY(cudaEventRecord(ev_panels, chain));
       // the columns updated next were last written by the previous group's side-stream launch
       if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
-      rank_update_kernel<<<dim3(kLook, nt), 256, 0, chain>>>(A, n, e, j0, kw, true);
+      rank_update_first_kernel<<<dim3(kLook, static_cast<unsigned>((n - e) / kNB)), 256, 0, chain>>>(A, n, e, j0, kw);
       rest_pending = false;
       if (has_rest) {
         ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_panels, 0));
-        rank_update_kernel<<<nt * (nt + 1), 256, 0, side>>>(A, n, e, j0, kw, false);
+        rank_update_kernel<<<nt * (nt + 1), 256, 0, side>>>(A, n, e, j0, kw);
         ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
         rest_pending = true;
       }
@@ -685,7 +758,7 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
   }
   for (int64_t s = 2 * kNB; s < n; s *= 2) {
     const unsigned pairs = static_cast<unsigned>((n + 2 * s - 1) / (2 * s));
-    const unsigned tiles = static_cast<unsigned>((s / kT) * (s / kTN));
+    const unsigned tiles = static_cast<unsigned>((s / kNB) * (s / kNB));
     merge1_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
     merge2_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
   }
