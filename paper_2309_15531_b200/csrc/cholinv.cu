@@ -28,6 +28,29 @@ constexpr int kGroup = 4;   // panels per rank-256 update
 
 __host__ __device__ __forceinline__ int64_t mn64(int64_t a, int64_t b) { return a < b ? a : b; }
 
+// Programmatic dependent launch for the chain of small kernels: a kernel launched with the
+// attribute below may be scheduled while its predecessor in the stream is still finishing; it then
+// waits here until that predecessor has completed and its writes are visible.  dep_release() lets
+// the successor of the calling kernel be scheduled early in the same way.  Both are no-ops for a
+// kernel launched the ordinary way.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // D += A B on 8 x 8 x 4 fp64 fragments: lane l holds A[l/4][l%4], B[l%4][l/4] and the two
 // outputs D[l/4][2 (l%4)], D[l/4][2 (l%4) + 1].
 __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
@@ -357,6 +380,8 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
   __shared__ double rdiag[kNB];          // 1 / L[j][j]
   const int tid = threadIdx.x;
   double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
+  dep_release();
+  dep_wait();
   {
     double v[kNB * kNB / 256];                         // all loads in flight before the first store
 #pragma unroll
@@ -499,6 +524,8 @@ panel_kernel(double* __restrict__ A, int64_t n, int k, const double* __restrict_
   TILE_SMEM
   const int64_t row0 = (static_cast<int64_t>(k) + 1 + blockIdx.x) * kNB;
   double* tile = A + row0 * n + static_cast<int64_t>(k) * kNB;
+  dep_release();
+  dep_wait();
   double acc[4][2][2] = {};
   tile_product<true>(tile, n, dinv + static_cast<int64_t>(k) * kNB * kNB, kNB, acc, sa, sb);
   for_each_pair64(acc, [&](int r, int c, const double* v) {
@@ -512,6 +539,8 @@ panel_kernel(double* __restrict__ A, int64_t n, int k, const double* __restrict_
 __global__ void __launch_bounds__(256)
 group_update_kernel(double* __restrict__ A, int64_t n, int k) {
   TILE_SMEM
+  dep_release();
+  dep_wait();
   if (blockIdx.y > blockIdx.x) return;
   const int64_t ri = (static_cast<int64_t>(k) + 1 + blockIdx.x) * kNB, rj = (static_cast<int64_t>(k) + 1 + blockIdx.y) * kNB;
   const int64_t ck = static_cast<int64_t>(k) * kNB;
@@ -539,6 +568,8 @@ __global__ void __launch_bounds__(256, 2)
 rank_update_first_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
   __shared__ TileSmem64 sm;
   const int ti = blockIdx.y, cj = blockIdx.x;               // 64-row block, 64-column block of the region
+  dep_release();
+  dep_wait();
   if (cj > ti) return;
   const int64_t ri = e + static_cast<int64_t>(ti) * kNB, rj = e + static_cast<int64_t>(cj) * kNB;
   if (rj >= n) return;
@@ -715,11 +746,11 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
   for (int g0 = 0; g0 < nb; g0 += kGroup) {
     const int g1 = g0 + kGroup < nb ? g0 + kGroup : nb;
     for (int k = g0; k < g1; ++k) {
-      potrf_kernel<<<1, 256, 0, chain>>>(A, n, k, dinv, status_dev);
+      ADADIM_CUDA_TRY(launch_chained(potrf_kernel, dim3(1), dim3(256), chain, A, n, k, dinv, status_dev));
       const int below = nb - k - 1;
-      if (below > 0) panel_kernel<<<below, 256, 0, chain>>>(A, n, k, dinv);
+      if (below > 0) ADADIM_CUDA_TRY(launch_chained(panel_kernel, dim3(below), dim3(256), chain, A, n, k, static_cast<const double*>(dinv)));
       const int inner = g1 - k - 1;
-      if (below > 0 && inner > 0) group_update_kernel<<<dim3(below, inner), 256, 0, chain>>>(A, n, k);
+      if (below > 0 && inner > 0) ADADIM_CUDA_TRY(launch_chained(group_update_kernel, dim3(below, inner), dim3(256), chain, A, n, k));
     }
     const int64_t e = static_cast<int64_t>(g1) * kNB;
     if (e < n) {
@@ -730,7 +761,7 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
       if (has_rest) ADADIM_CUDA_TRY(cudaEventRecord(ev_panels, chain));
       // the columns updated next were last written by the previous group's side-stream launch
       if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
-      rank_update_first_kernel<<<dim3(kLook, static_cast<unsigned>((n - e) / kNB)), 256, 0, chain>>>(A, n, e, j0, kw);
+      ADADIM_CUDA_TRY(launch_chained(rank_update_first_kernel, dim3(kLook, static_cast<unsigned>((n - e) / kNB)), dim3(256), chain, A, n, e, j0, kw));
       rest_pending = false;
       if (has_rest) {
         ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_panels, 0));
