@@ -28,6 +28,8 @@ if ROOT not in sys.path:
 
 METRIC = "AdaDim layer quant weights/s (RTN & GPTQ, 3b g128); % of HBM/tensor roofline"
 BITS, GROUP = 3, 128
+WORKLOAD = ("llama7b_q_proj W[4096,4096] fp16, X[262144,4096] bf16, 3-bit g128, "
+            "Hessian + RTN both dims + score + factor + GPTQ both dims + score")
 
 
 def _peaks():
@@ -352,8 +354,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "llama7b_q_proj W[4096,4096] fp16, X[262144,4096] bf16, 3-bit g128, "
-                               "Hessian + RTN both dims + score + factor + GPTQ both dims + score",
+        "config": {"workload": WORKLOAD,
                    "l2": "flushed between steps by writing a 256 MiB buffer; X (2.1 GB) exceeds L2",
                    "replicas": world},
         "stages_ms": stage_ms,
@@ -424,8 +425,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": args.gpus,
             "steps": n, "warmup": 1, "ms_per_step": 4096 * 4096 / value * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "llama7b_q_proj W[4096,4096] fp16, X[262144,4096] bf16, 3-bit g128 (CPU oracle, "
-                                   "bounded sample scaled to the full layer)"},
+            "config": {"workload": WORKLOAD, "l2": "not applicable: CPU oracle on a bounded sample scaled to the full layer",
+                       "replicas": 1},
             "cpu_baseline": last,
             "e2e": {"value": value, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
