@@ -397,46 +397,49 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
   }
   __syncthreads();
 
-#pragma unroll 1
-  for (int j0 = 0; j0 < kNB; j0 += kSub) {
-    // (a) the 8 x 8 diagonal piece, in every thread of the two warps that own the rows below
-    double d[kSub][kSub], rinv[kSub];
-    const int row = j0 + kSub + tid;                   // the row below that this thread solves
-    double x[kSub];
-    bool bad = false;
-    if (tid < 64) {
+  // Sub-panel j's factor-and-solve (a) depends only on the next eight columns of the block.  After
+  // each sub-panel the two warps that run (a) therefore update just those columns (b1) and go
+  // straight on to the next (a), while the other six warps update the rest of the block (b2).
+  double d[kSub][kSub], rinv[kSub], x[kSub];
+  bool bad = false;
+  // (a): the 8 x 8 diagonal piece at j0, factored in registers by every thread of warps 0 and 1,
+  // and the thread's row below it solved by substitution (finished entries pushed forward)
+  auto factor_and_solve = [&](int j0) {
+    const int row = j0 + kSub + tid;
 #pragma unroll
-      for (int r = 0; r < kSub; ++r)
+    for (int r = 0; r < kSub; ++r)
 #pragma unroll
-        for (int c = 0; c <= r; ++c) d[r][c] = M[j0 + r][j0 + c];
-      if (row < kNB) {
+      for (int c = 0; c <= r; ++c) d[r][c] = M[j0 + r][j0 + c];
+    if (row < kNB) {
 #pragma unroll
-        for (int c = 0; c < kSub; ++c) x[c] = M[row][j0 + c];
-      }
+      for (int c = 0; c < kSub; ++c) x[c] = M[row][j0 + c];
+    }
+#pragma unroll
+    for (int c = 0; c < kSub; ++c) {
+      double piv = d[c][c];
+      if (!(piv > 0.0)) { bad = true; piv = 1.0; }
+      const double r = rsqrt(piv);
+      rinv[c] = r;
+      d[c][c] = piv * r;
+#pragma unroll
+      for (int r2 = c + 1; r2 < kSub; ++r2) d[r2][c] *= r;
+#pragma unroll
+      for (int c2 = c + 1; c2 < kSub; ++c2)
+#pragma unroll
+        for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
+    }
+    if (row < kNB) {
 #pragma unroll
       for (int c = 0; c < kSub; ++c) {
-        double piv = d[c][c];
-        if (!(piv > 0.0)) { bad = true; piv = 1.0; }
-        const double r = rsqrt(piv);
-        rinv[c] = r;
-        d[c][c] = piv * r;
+        x[c] *= rinv[c];
 #pragma unroll
-        for (int r2 = c + 1; r2 < kSub; ++r2) d[r2][c] *= r;
-#pragma unroll
-        for (int c2 = c + 1; c2 < kSub; ++c2)
-#pragma unroll
-          for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
-      }
-      if (row < kNB) {                               // x D^T = a by substitution, finished entries pushed forward
-#pragma unroll
-        for (int c = 0; c < kSub; ++c) {
-          x[c] *= rinv[c];
-#pragma unroll
-          for (int c2 = c + 1; c2 < kSub; ++c2) x[c2] = fma(-x[c], d[c2][c], x[c2]);
-        }
+        for (int c2 = c + 1; c2 < kSub; ++c2) x[c2] = fma(-x[c], d[c2][c], x[c2]);
       }
     }
-    __syncthreads();                                   // every thread has read the old piece
+  };
+  // results of (a) at j0 into M: each row owner its row, one thread the diagonal piece
+  auto write_back = [&](int j0) {
+    const int row = j0 + kSub + tid;
     if (row < kNB) {
 #pragma unroll
       for (int c = 0; c < kSub; ++c) M[row][j0 + c] = x[c];
@@ -449,31 +452,63 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
       }
       if (bad) report(status_dev, ADADIM_ERR_NOT_PD);
     }
-    __syncthreads();
-    // (b) M[r][c] -= sum_m M[r][j0+m] M[c][j0+m] for lim <= c <= r; thread (ty, tx) owns rows
-    // ty + 16 i and columns tx + 16 j (neighbouring lanes read neighbouring rows: no bank conflicts)
+  };
+
+  if (tid < 64) factor_and_solve(0);
+  __syncthreads();                                     // every thread has read the old piece
+  if (tid < 64) write_back(0);
+  __syncthreads();
+#pragma unroll 1
+  for (int j0 = 0; j0 + kSub < kNB; j0 += kSub) {
     const int lim = j0 + kSub;
-    if (lim < kNB) {
-      const int tx = tid & 15, ty = tid >> 4;
-      double acc[4][4] = {};
+    if (tid < 64) {
+      // (b1) M[r][lim + c] -= sum_m M[r][j0+m] M[lim+c][j0+m] for the next eight columns, one row per thread
+      const int r = lim + tid;
+      if (r < kNB) {
+        double am[kSub], acc[kSub];
 #pragma unroll
-      for (int m = 0; m < kSub; ++m) {
-        double a[4], b[4];
+        for (int m = 0; m < kSub; ++m) am[m] = M[r][j0 + m];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { a[i] = M[ty + 16 * i][j0 + m]; b[i] = M[tx + 16 * i][j0 + m]; }
+        for (int c = 0; c < kSub; ++c) {
+          acc[c] = 0.0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int r = ty + 16 * i, c = tx + 16 * j;
-          if (c >= lim && c <= r) M[r][c] -= acc[i][j];
+          for (int m = 0; m < kSub; ++m) acc[c] = fma(am[m], M[lim + c][j0 + m], acc[c]);
         }
+#pragma unroll
+        for (int c = 0; c < kSub; ++c)
+          if (lim + c <= r) M[r][lim + c] -= acc[c];
+      }
+      asm volatile("bar.sync 1, 64;" ::: "memory");    // warps 0 and 1 only
+      factor_and_solve(lim);
+    } else {
+      // (b2) the same update for the columns after those, lim + 8 <= c <= r, on the other 192 threads:
+      // thread (ty, tx) owns rows ty + 12 i and columns tx + 16 j
+      const int t2 = tid - 64, tx = t2 & 15, ty = t2 >> 4;
+      if (lim + kSub < kNB) {
+        double acc[6][4] = {};
+#pragma unroll
+        for (int m = 0; m < kSub; ++m) {
+          double av[6], bv[4];
+#pragma unroll
+          for (int i = 0; i < 6; ++i) av[i] = ty + 12 * i < kNB ? M[ty + 12 * i][j0 + m] : 0.0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) bv[j] = M[tx + 16 * j][j0 + m];
+#pragma unroll
+          for (int i = 0; i < 6; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 6; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int r = ty + 12 * i, c = tx + 16 * j;
+            if (r < kNB && c >= lim + kSub && c <= r) M[r][c] -= acc[i][j];
+          }
+      }
     }
+    __syncthreads();                                   // (b2) done; every thread of (a) has read its inputs
+    if (tid < 64) write_back(lim);
     __syncthreads();
   }
 
