@@ -236,22 +236,38 @@ block_kernel(const BlockArgs a) {
   const int64_t row = row0 + tid;
   float* Wd = a.Wc + static_cast<int64_t>(d) * a.out * a.in;
 
-  // stage the slab and the U block (coalesced), then work row-per-thread; eight rows' worth of
-  // loads are in flight before the first is stored, so the copy costs 4 memory latencies, not 32
+  // Stage the U block and the slab (coalesced), then work row-per-thread; eight rows' worth of
+  // loads are in flight before the first is stored, so each copy costs 4 memory latencies, not 32.
+  // The kernel may have been scheduled while the launch before it in the stream (the update of this
+  // block's columns) is still finishing: U does not depend on it and is staged first; everything
+  // after the wait sees that launch's results.
 #pragma unroll 1
   for (int e0 = 0; e0 < kBlk * kBlk / 4; e0 += 8 * kBlk) {
-    float4 wv[8], uv[8];
+    float4 uv[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
-      wv[u] = *reinterpret_cast<const float4*>(Wd + (row0 + r) * a.in + a.i1 + c4);
       uv[u] = *reinterpret_cast<const float4*>(a.U + static_cast<int64_t>(a.i1 + r) * a.in + a.i1 + c4);
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
-      Ws[r * kPad + c4 + 0] = wv[u].x; Ws[r * kPad + c4 + 1] = wv[u].y; Ws[r * kPad + c4 + 2] = wv[u].z; Ws[r * kPad + c4 + 3] = wv[u].w;
       *reinterpret_cast<float4*>(Us + r * kBlk + c4) = uv[u];
+    }
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#pragma unroll 1
+  for (int e0 = 0; e0 < kBlk * kBlk / 4; e0 += 8 * kBlk) {
+    float4 wv[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
+      wv[u] = *reinterpret_cast<const float4*>(Wd + (row0 + r) * a.in + a.i1 + c4);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
+      Ws[r * kPad + c4 + 0] = wv[u].x; Ws[r * kPad + c4 + 1] = wv[u].y; Ws[r * kPad + c4 + 2] = wv[u].z; Ws[r * kPad + c4 + 3] = wv[u].w;
     }
   }
   __syncthreads();
@@ -412,7 +428,19 @@ template <int BITS, int G>
 int block_launch(const BlockArgs& a, int slabs, int ndim, cudaStream_t st) {
   ADADIM_CUDA_TRY(cudaFuncSetAttribute(block_kernel<BITS, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(block_smem_bytes())));
-  block_kernel<BITS, G><<<dim3(slabs, ndim), kBlk, block_smem_bytes(), st>>>(a);
+  // launched so that it may be scheduled while the kernel before it in the stream finishes
+  // (it waits for that kernel itself, after staging what does not depend on it)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(slabs, ndim);
+  cfg.blockDim = dim3(kBlk);
+  cfg.dynamicSmemBytes = block_smem_bytes();
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ADADIM_CUDA_TRY(cudaLaunchKernelEx(&cfg, block_kernel<BITS, G>, a));
   return ADADIM_OK;
 }
 

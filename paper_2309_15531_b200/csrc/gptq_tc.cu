@@ -65,6 +65,9 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // a kernel launched behind this one with programmatic serialization may be scheduled from now
+  // on; it still waits for this grid's completion before it reads anything this grid writes
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // this CTA's tiles: an even share of [0, ntiles)
   const int per = (p.ntiles + gridDim.x - 1) / gridDim.x;
   const int t0 = blockIdx.x * per;
