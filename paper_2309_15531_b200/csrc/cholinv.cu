@@ -64,29 +64,31 @@ __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
 // Each of the eight warps owns 32 rows x 16 columns as 4 x 2 fragments.  These tiles sit on the
 // factorization's critical chain, so every global load of both operands is issued before the
 // first one is used (one memory latency per tile), and the operands are staged in two K-halves.
-// The row pitch is 8 mod 16 doubles: a fragment's 4 k-rows x 8 columns fall on distinct banks.
+// The row pitch is 4 mod 16 doubles: 64-bit shared-memory accesses are served a half-warp at a
+// time, and a half-warp's fragment load (4 k-rows x 4 columns) then falls on 16 distinct banks;
+// the loaders put consecutive lanes on consecutive rows, so their transposing stores do too.
 constexpr int kHalfK = kNB / 2;
 #define TILE_SMEM                           \
-  __shared__ double sa[kHalfK][kNB + 8];    \
-  __shared__ double sb[kHalfK][kNB + 8];
+  __shared__ double sa[kHalfK][kNB + 4];    \
+  __shared__ double sb[kHalfK][kNB + 4];
 
 template <bool B_T>
 __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64_t lda, const double* __restrict__ B,
-                                             int64_t ldb, double (&acc)[4][2][2], double (*sa)[kNB + 8],
-                                             double (*sb)[kNB + 8]) {
+                                             int64_t ldb, double (&acc)[4][2][2], double (*sa)[kNB + 4],
+                                             double (*sb)[kNB + 4]) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = (warp & 1) * 32, wn = (warp >> 1) * 16;
   const int fk = lane & 3, fr = lane >> 2;
-  const int r = tid >> 2, kq = (tid & 3) * 8;            // loader: row (or column of B^T), first k of eight
-  const int kk = tid >> 3, nq = (tid & 7) * 8;           // loader of a non-transposed B: k row, first column of eight
+  const int r = tid & 63, kq = (tid >> 6) * 8;           // loader: row (or column of B^T), first k of eight
+  const int kk = tid >> 3, nc = tid & 7;                 // loader of a non-transposed B: k row, 16-byte chunks nc + 8 t
   double2 av[2][4], bv[2][4];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const double2* asrc = reinterpret_cast<const double2*>(A + static_cast<int64_t>(r) * lda + h * kHalfK + kq);
     const double2* bsrc = B_T ? reinterpret_cast<const double2*>(B + static_cast<int64_t>(r) * ldb + h * kHalfK + kq)
-                              : reinterpret_cast<const double2*>(B + static_cast<int64_t>(h * kHalfK + kk) * ldb + nq);
+                              : reinterpret_cast<const double2*>(B + static_cast<int64_t>(h * kHalfK + kk) * ldb) + nc;
 #pragma unroll
-    for (int t = 0; t < 4; ++t) { av[h][t] = asrc[t]; bv[h][t] = bsrc[t]; }
+    for (int t = 0; t < 4; ++t) { av[h][t] = asrc[t]; bv[h][t] = bsrc[B_T ? t : 8 * t]; }
   }
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
@@ -95,7 +97,7 @@ __device__ __forceinline__ void tile_product(const double* __restrict__ A, int64
     for (int t = 0; t < 4; ++t) {
       sa[kq + 2 * t][r] = av[h][t].x; sa[kq + 2 * t + 1][r] = av[h][t].y;
       if (B_T) { sb[kq + 2 * t][r] = bv[h][t].x; sb[kq + 2 * t + 1][r] = bv[h][t].y; }
-      else *reinterpret_cast<double2*>(&sb[kk][nq + 2 * t]) = bv[h][t];
+      else *reinterpret_cast<double2*>(&sb[kk][2 * (nc + 8 * t)]) = bv[h][t];
     }
     __syncthreads();
 #pragma unroll
@@ -131,12 +133,12 @@ __device__ __forceinline__ void for_each_pair64(double (&acc)[4][2][2], F f) {
 // bandwidth here).  Rows >= a_rows (64 or 128) of A are not read (treated as zero).  K is a
 // multiple of 8.  Shared-memory slabs are double-buffered; the slab after the next one is already
 // on its way from global memory into registers while the current one is multiplied, and two CTAs
-// share an SM, so global latency is covered.  The row pitches are 8 mod 16 doubles: the 4 k-rows
-// x 8 columns of a fragment load then fall on distinct banks.
+// share an SM, so global latency is covered.  The row pitches are 4 mod 16 doubles and the
+// loaders put consecutive lanes on consecutive rows (see tile_product): no bank conflicts.
 constexpr int kT = 128, kTN = 64, kBK = 8;
 struct TileSmem {
-  double a[2][kBK][kT + 8];
-  double b[2][kBK][kTN + 8];
+  double a[2][kBK][kT + 4];
+  double b[2][kBK][kTN + 4];
 };
 
 // acc[i][j] is the fragment at rows 8 i, columns 8 j of the warp's piece: this lane holds row
@@ -148,8 +150,8 @@ __device__ __forceinline__ void product_tile(const double* __restrict__ A, int64
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = (warp & 3) * 32, wn = (warp >> 2) * 32;
   const int fk = lane & 3, fr = lane >> 2;                      // fragment coordinates of this lane
-  const int ar = tid >> 1, akq = (tid & 1) * 4;                 // A loader: row, first k of four
-  const int br = tid >> 2, bkq = (tid & 3) * 2;                 // B loader (transposed): column, first k of two
+  const int ar = tid & 127, akq = (tid >> 7) * 4;               // A loader: row, first k of four
+  const int br = tid & 63, bkq = (tid >> 6) * 2;                // B loader (transposed): column, first k of two
   const int bkk = tid >> 5, bnq = (tid & 31) * 2;               // B loader (not transposed): k row, first col of two
   const bool a_ok = ar < a_rows;
   const double* ap = A + static_cast<int64_t>(ar) * lda + akq;
@@ -223,8 +225,8 @@ __device__ __forceinline__ void for_each_pair(double (&acc)[4][4][2], F f) {
 // columns; the merges, whose longest reductions decide the kernel's length): half the work per
 // CTA, twice the CTAs.  Warps own 32 x 16 pieces (4 x 2 fragments) as in tile_product.
 struct TileSmem64 {
-  double a[2][kBK][kNB + 8];
-  double b[2][kBK][kNB + 8];
+  double a[2][kBK][kNB + 4];
+  double b[2][kBK][kNB + 4];
 };
 
 template <bool B_T>
@@ -234,7 +236,7 @@ __device__ __forceinline__ void product_tile64(const double* __restrict__ A, int
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = (warp & 1) * 32, wn = (warp >> 1) * 16;
   const int fk = lane & 3, fr = lane >> 2;
-  const int ar = tid >> 2, akq = (tid & 3) * 2;                 // A / B^T loader: row, first k of two
+  const int ar = tid & 63, akq = (tid >> 6) * 2;                // A / B^T loader: row, first k of two
   const int bkk = tid >> 5, bnq = (tid & 31) * 2;               // B loader (not transposed): k row, first col of two
   const double* ap = A + static_cast<int64_t>(ar) * lda + akq;
   const double* bp = B_T ? B + static_cast<int64_t>(ar) * ldb + akq : B + static_cast<int64_t>(bkk) * ldb + bnq;
