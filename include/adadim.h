@@ -103,7 +103,7 @@ ADADIM_API int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_to
  *     z  = clamp(rint(-lo / s), 0, maxq)
  *     c  = clamp(rint(w / s) + z, 0, maxq)          maxq = 2^bits - 1, rint = ties to even
  *   W      [out][in], wdtype ADADIM_F16 or ADADIM_F32; ldw in elements, 16-byte aligned rows.
- *   bits   3 or 4;  group 32, 64 or 128.
+ *   bits   3 or 4;  group 32, 64, 128 or 256 (the paper's sweep, Section 4.4, uses 64, 128, 256).
  *   dim    ADADIM_DIM_OC (q_oc written), ADADIM_DIM_IC (q_ic written) or ADADIM_DIM_BOTH.
  *   Shape rules: in % 32 == 0; per-OC needs in % group == 0; per-IC needs out % group == 0.
  *   out == 0 or in == 0 is accepted and does nothing.
@@ -136,7 +136,8 @@ ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, float 
  *   H          [in][in] fp32, required: its diagonal marks the dead columns, and when U == NULL
  *              the factor is computed from it into workspace.
  *   U          optional precomputed adadim_cholesky_inverse_factor of the same H, or NULL.
- *   blocksize  128.  group must divide 128.  in % 128 == 0, out % 128 == 0.
+ *   blocksize  128.  group must divide 128 (32, 64, 128; 256 is refused with ADADIM_ERR_PARAM).
+ *              in % 128 == 0, out % 128 == 0.
  *   gptq_loss  optional device double[2] (OC, IC): 1/2 * sum of e^2.
  *   workspace  adadim_workspace_bytes(ADADIM_WS_GPTQ, out, in, bits, group), 256-byte aligned.
  */

@@ -31,9 +31,11 @@ int check_weight(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
   return ADADIM_OK;
 }
 
-int check_quant_params(int bits, int group) {
+// group 256 is accepted by the round-to-nearest quantizer and the scorer; GPTQ works in
+// 128-column blocks on 128-row slabs and takes groups that divide 128
+int check_quant_params(int bits, int group, bool allow_256) {
   if (bits != 3 && bits != 4) return ADADIM_ERR_PARAM;
-  if (group != 32 && group != 64 && group != 128) return ADADIM_ERR_PARAM;
+  if (group != 32 && group != 64 && group != 128 && !(allow_256 && group == 256)) return ADADIM_ERR_PARAM;
   return ADADIM_OK;
 }
 
@@ -112,7 +114,7 @@ int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_tokens, int64
 int adadim_quantize_rtn(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, int bits, int group, int dim,
                         const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group);
+  int rc = check_quant_params(bits, group, true);
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (out < 0 || in < 0) return ADADIM_ERR_SHAPE;
@@ -148,7 +150,7 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* gptq_loss, int* status_dev,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group);
+  int rc = check_quant_params(bits, group, false);
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
@@ -176,7 +178,7 @@ int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64
                                    int32_t* perm_out, int* status_dev, void* workspace, size_t workspace_bytes,
                                    void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group);
+  int rc = check_quant_params(bits, group, false);
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
@@ -202,7 +204,7 @@ int adadim_score_select(const void* W, int wdtype, int64_t out, int64_t in, int6
                         int group, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* err, int* chosen,
                         int* status_dev, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group);
+  int rc = check_quant_params(bits, group, true);
   if (rc != ADADIM_OK) return rc;
   if (out <= 0 || in <= 0) return ADADIM_ERR_SHAPE;
   rc = check_weight(W, wdtype, out, in, ldw);

@@ -466,6 +466,132 @@ void launch_group_half(const __half* W, int64_t out, int64_t in, int64_t ldw, in
   else launch_dims<BITS, 32>(W, out, in, ldw, dim, qoc, qic, st);
 }
 
+// ---- g = 256 (the largest group size of the paper's sweep, Section 4.4) ------------------------
+// A 256 x 256 tile holds whole groups of both dimensions but not in registers, so the tile is read
+// twice: once for the statistics, once (from L2, where it still is) for the codes.  A warp covers
+// one row of the tile per pass (32 lanes x 8 columns), so a per-OC group is one warp-wide
+// reduction; per-IC statistics are accumulated per thread over the 32 passes and combined across
+// the eight warps through shared memory.  Exact formula throughout (the general quotient).
+constexpr int kTile256 = 256;
+template <typename T, int BITS, bool DO_OC, bool DO_IC>
+__global__ void __launch_bounds__(kThreads, 2)
+rtn_g256_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, adadim_qtensor qoc, adadim_qtensor qic) {
+  constexpr float maxq = static_cast<float>((1 << BITS) - 1);
+  constexpr float rcp_maxq = 1.0f / maxq;
+  constexpr int kRowsPerPass = kThreads / 32;            // 8
+  constexpr int kPasses256 = kTile256 / kRowsPerPass;    // 32
+  __shared__ float s_cmn[kRowsPerPass][kTile256], s_cmx[kRowsPerPass][kTile256];
+  __shared__ float s_ic_s[kTile256], s_ic_r[kTile256];
+  __shared__ int s_ic_nb[kTile256];
+  __shared__ float s_oc_s[kTile256], s_oc_r[kTile256];
+  __shared__ int s_oc_nb[kTile256];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kTile256, c0 = static_cast<int64_t>(blockIdx.x) * kTile256;
+  const int64_t col = c0 + lane * 8;
+  const bool col_ok = col < in;
+  const int64_t words_per_row = in * BITS / 32;
+
+  // ---- statistics ----------------------------------------------------------------------------
+  float cmn[8], cmx[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) { cmn[k] = 0.0f; cmx[k] = 0.0f; }    // 0 always lies inside [lo, hi]
+#pragma unroll 4
+  for (int p = 0; p < kPasses256; ++p) {
+    const int lr = p * kRowsPerPass + warp;
+    const int64_t row = r0 + lr;
+    float w[8];
+    if (col_ok && row < out) load8(W + row * ldw + col, w);
+    else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) w[k] = 0.0f;
+    }
+    if (DO_IC) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { cmn[k] = fminf(cmn[k], w[k]); cmx[k] = fmaxf(cmx[k], w[k]); }
+    }
+    if (DO_OC) {
+      float mn = w[0], mx = w[0];
+#pragma unroll
+      for (int k = 1; k < 8; ++k) { mn = fminf(mn, w[k]); mx = fmaxf(mx, w[k]); }
+#pragma unroll
+      for (int m = 16; m > 0; m >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, m));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+      }
+      if (lane == 0) {
+        const GroupParams gp = group_params(mn, mx, maxq, rcp_maxq);
+        s_oc_s[lr] = gp.s; s_oc_r[lr] = gp.rcp; s_oc_nb[lr] = static_cast<int>(gp.z) - kRoundMagicBits;
+        if (row < out && c0 < in) {
+          const int64_t idx = row * (in / kTile256) + c0 / kTile256;
+          qoc.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
+          qoc.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
+        }
+      }
+    }
+  }
+  if (DO_IC) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { s_cmn[warp][lane * 8 + k] = cmn[k]; s_cmx[warp][lane * 8 + k] = cmx[k]; }
+  }
+  __syncthreads();
+  if (DO_IC) {
+    const int c = tid;                                   // one column per thread
+    float mn = s_cmn[0][c], mx = s_cmx[0][c];
+#pragma unroll
+    for (int wv = 1; wv < kRowsPerPass; ++wv) { mn = fminf(mn, s_cmn[wv][c]); mx = fmaxf(mx, s_cmx[wv][c]); }
+    const GroupParams gp = group_params(mn, mx, maxq, rcp_maxq);
+    s_ic_s[c] = gp.s; s_ic_r[c] = gp.rcp; s_ic_nb[c] = static_cast<int>(gp.z) - kRoundMagicBits;
+    const int64_t grow = r0 / kTile256;
+    if (c0 + c < in && r0 < out) {
+      qic.scales[grow * in + c0 + c] = __half_as_ushort(__float2half_rn(gp.s));
+      qic.zeros[grow * in + c0 + c] = __half_as_ushort(__float2half_rn(gp.z));
+    }
+  }
+  __syncthreads();
+
+  // ---- codes ---------------------------------------------------------------------------------
+  float ic_s[8], ic_r[8];
+  int ic_nb[8];
+  if (DO_IC) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { ic_s[k] = s_ic_s[lane * 8 + k]; ic_r[k] = s_ic_r[lane * 8 + k]; ic_nb[k] = s_ic_nb[lane * 8 + k]; }
+  }
+#pragma unroll 2
+  for (int p = 0; p < kPasses256; ++p) {
+    const int lr = p * kRowsPerPass + warp;
+    const int64_t row = r0 + lr;
+    const bool ok = col_ok && row < out;
+    float w[8];
+    if (ok) load8(W + row * ldw + col, w);
+    else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) w[k] = 0.0f;
+    }
+    if (DO_OC) {
+      float s8[8], r8[8];
+      int nb8[8];
+      const float sv = s_oc_s[lr], rv = s_oc_r[lr];
+      const int nbv = s_oc_nb[lr];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { s8[k] = sv; r8[k] = rv; nb8[k] = nbv; }
+      store_codes<BITS>(pack8<BITS>(w, s8, r8, nb8), qoc.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, lane, ok);
+    }
+    if (DO_IC) {
+      store_codes<BITS>(pack8<BITS>(w, ic_s, ic_r, ic_nb), qic.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, lane, ok);
+    }
+  }
+}
+
+template <typename T, int BITS>
+void launch_g256(const T* W, int64_t out, int64_t in, int64_t ldw, int dim,
+                 const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  dim3 grid(static_cast<unsigned>((in + kTile256 - 1) / kTile256), static_cast<unsigned>((out + kTile256 - 1) / kTile256));
+  if (dim == ADADIM_DIM_BOTH) rtn_g256_kernel<T, BITS, true, true><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+  else if (dim == ADADIM_DIM_OC) rtn_g256_kernel<T, BITS, true, false><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+  else rtn_g256_kernel<T, BITS, false, true><<<grid, kThreads, 0, st>>>(W, out, in, ldw, qoc, qic);
+}
+
 template <int BITS>
 __global__ void unpack_kernel(const uint32_t* __restrict__ codes, int64_t out, int64_t in, uint8_t* __restrict__ dst) {
   // one thread per 32 codes (BITS words of input, 32 bytes of output)
@@ -496,6 +622,16 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ codes, int64_t out, i
 
 int rtn_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, int bits, int group, int dim,
                const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  if (group == 256) {
+    if (wdtype == ADADIM_F16) {
+      if (bits == 3) launch_g256<__half, 3>(static_cast<const __half*>(W), out, in, ldw, dim, qoc, qic, st);
+      else launch_g256<__half, 4>(static_cast<const __half*>(W), out, in, ldw, dim, qoc, qic, st);
+    } else {
+      if (bits == 3) launch_g256<float, 3>(static_cast<const float*>(W), out, in, ldw, dim, qoc, qic, st);
+      else launch_g256<float, 4>(static_cast<const float*>(W), out, in, ldw, dim, qoc, qic, st);
+    }
+    return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+  }
   if (wdtype == ADADIM_F16) {
     if (bits == 3) launch_group_half<3>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
     else launch_group_half<4>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);

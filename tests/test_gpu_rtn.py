@@ -96,3 +96,49 @@ def test_empty_and_bad_arguments():
     with pytest.raises(B.AdadimError) as e:                  # misaligned rows
         B.quantize_rtn(torch.zeros(128, 132, dtype=torch.float16, device="cuda")[:, 4:], 3, 128, B.DIM_OC)
     assert e.value.status == 5
+
+
+# ----------------------------------------------------------------------------- g = 256 (Section 4.4 sweep)
+
+@pytest.mark.parametrize("bits", [3, 4])
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+def test_group_256(bits, dtype):
+    W = I.make_weight(I.WeightSpec(768, 1024, dtype, 0.02, 0.005, seed=83), "cuda")
+    W[3, :] *= 15.0
+    W[:, 700] *= 25.0
+    _check_both(W, bits, 256)
+
+
+def test_group_256_special_groups_and_partial_tiles():
+    W = I.make_weight(I.WeightSpec(512, 768, "f32", 0.02, 0.0, seed=84), "cuda")
+    W[0:256, 0:256] = 0.0                                   # all-zero groups in both dimensions
+    W[256:512, 0:256] = W[256:512, 0:256].abs() + 0.01      # one-signed
+    W[300, 600] = 3.0e6                                     # range overflows fp16
+    _check_both(W, 3, 256)
+    # per-IC only needs out % 256 == 0: the column tiles may be partial (in % 32 == 0)
+    V = I.make_weight(I.WeightSpec(256, 416, "f16", 0.02, 0.0, seed=85), "cuda")
+    _, q_ic = B.quantize_rtn(V, 4, 256, B.DIM_IC)
+    torch.cuda.synchronize()
+    assert_rtn_equal(q_ic, O.quantize_rtn(to_np(V).astype(np.float32), 4, 256, "ic"), "ic b4 g256 partial")
+
+
+def test_group_256_selection_flow():
+    """RTN in both dimensions at g = 256, scored and selected: the setting where the paper reports
+    the largest gain of the adaptive choice over plain RTN (Section 4.4)."""
+    from paper_2309_15531_b200 import flows
+    W = I.make_weight(I.WeightSpec(512, 512, "f16", 0.02, 0.0, seed=86), "cuda")
+    X = I.make_calib(I.CalibSpec(2048, 512, "bf16", "normal", 3, 50.0, 100.0, seed=87), "cuda")
+    W[:, :8] *= 0.1
+    Hn = O.hessian(to_np(X)).astype(np.float32)
+    dim, err, _ = flows.rtn_ada(W, torch.as_tensor(Hn, device="cuda"), 3, 256)
+    torch.cuda.synchronize()
+    best, ref, _ = O.rtn_ada(to_np(W).astype(np.float32), Hn.astype(np.float64), 3, 256)
+    assert B.DIM_NAMES[dim] == best
+    assert err[0].item() == pytest.approx(ref["oc"], rel=1e-3) and err[1].item() == pytest.approx(ref["ic"], rel=1e-3)
+
+
+def test_gptq_refuses_group_256():
+    W = I.make_weight(I.WeightSpec(256, 256, "f16", 0.02, 0.0, seed=88), "cuda")
+    H = 2.0 * torch.eye(256, device="cuda")
+    with pytest.raises(Exception):
+        B.quantize_gptq(W, H, 3, 256, B.DIM_BOTH)
