@@ -170,3 +170,21 @@ def test_reordered_full_size_layer():
         D = torch.as_tensor(Wn.astype(np.float64) - O.dequantize(codes, s, z, 128, name).astype(np.float64), device="cuda")
         tr = 0.5 * float(((D @ Hd_t) * D).sum().item())
         assert loss[k] == pytest.approx(tr, rel=1e-3)
+
+
+def test_row_pitch_and_fp32_weights():
+    """A view with a row pitch larger than its width (the gather of the working copies and the static
+    parameters read W through ldw) and fp32 weights give the same result as a dense fp32 copy."""
+    full = I.make_weight(I.WeightSpec(256, 512, "f32", 0.02, 0.0, seed=72), "cuda")
+    Wv = full[:, :384]                                       # pitch 512, width 384
+    Wd = Wv.contiguous()
+    X = I.make_calib(I.CalibSpec(2048, 384, "f32", "normal", 2, 30.0, 60.0, seed=73), "cuda")
+    Hn = O.hessian(to_np(X)).astype(np.float32)
+    a_oc, a_ic, la, pa = _run(Wv, Hn, 3, 128)
+    b_oc, b_ic, lb, pb = _run(Wd, Hn, 3, 128)
+    assert np.array_equal(pa, pb) and np.array_equal(la, lb)
+    for a, b in ((a_oc, b_oc), (a_ic, b_ic)):
+        assert torch.equal(a.codes, b.codes) and torch.equal(a.scales, b.scales) and torch.equal(a.zeros, b.zeros)
+    ref = O.quantize_gptq_reordered(to_np(Wd), Hn, 3, 128, "ic", 0.01)
+    frac, lvl = code_mismatch(q_to_np(a_ic)[0], ref["codes"])
+    assert frac <= 1e-3 and lvl <= 1
