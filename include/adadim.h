@@ -22,8 +22,11 @@
  *     into it, so to the caller these calls are ordered on `cuda_stream` like the others.
  *   - The return value is an adadim_status.  Argument errors are found on the host before
  *     anything is launched.  Conditions only the device can see (a non-positive Cholesky
- *     pivot, a wait that ran out) are written to the caller's `status_dev` word, which the
- *     call first sets to ADADIM_OK; kernels never trap.
+ *     pivot, a NaN error, a wait that ran out) are written to the caller's `status_dev` word;
+ *     kernels never trap.  The word is STICKY: the caller sets it to ADADIM_OK (0) once, may
+ *     pass the same word to any sequence of calls, and reads it when convenient; a call only
+ *     ever changes it from ADADIM_OK to the first condition it meets and never clears it, so
+ *     an early call's error survives the later calls.
  *   - Non-finite weights or activations give unspecified codes (no error is raised).
  */
 #ifndef ADADIM_H_
@@ -116,12 +119,14 @@ ADADIM_API int adadim_quantize_rtn(const void* W, int wdtype, int64_t out, int64
  * Damped Cholesky-inverse factor used by GPTQ (Section 2.2; the damping is the published
  * algorithm's): columns with H[i,i] == 0 get H[i,i] = 1 ("dead" columns), then
  *     Hd = H + lambda*I,  lambda = percdamp * mean(diag H),   U upper triangular, Hd^-1 = U^T U.
- *   H  [in][in] fp32 (not modified);  U [in][in] fp32 out, strictly-lower part set to 0.
+ *   H  [in][in] fp32 (not modified);  U [in][in] fp64 out, strictly-lower part set to 0.
+ *      (U is binary64 because GPTQ's rounding decisions thousands of columns later depend on
+ *      it: see adadim_quantize_gptq.)
  *   in must be a multiple of 64.
  *   workspace  adadim_workspace_bytes(ADADIM_WS_FACTOR, 0, in, 0, 0) bytes, 256-byte aligned.
  *   status_dev ADADIM_ERR_NOT_PD if a pivot is not positive.
  */
-ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, float percdamp, float* U,
+ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, double percdamp, double* U,
                                    int* status_dev, void* workspace, size_t workspace_bytes,
                                    void* cuda_stream);
 
@@ -133,6 +138,11 @@ ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, float 
  * (already compensated) weights with the formula of adadim_quantize_rtn: per-OC at each
  * group's first column, from that group's columns; per-IC at every column, from its g-row
  * groups.  Weights of dead columns are treated as 0.
+ * Precision: the working weights, U and every error and update are binary64; the weight as it
+ * stands when its column is reached is rounded once to binary32 and quantized with the binary32
+ * formula above.  (A binary32 working copy drifts by a few 1e-6 of a quantization step over
+ * thousands of columns, which is enough to flip individual roundings, and every flip changes
+ * all later columns of its row or group.)
  *   H          [in][in] fp32, required: its diagonal marks the dead columns, and when U == NULL
  *              the factor is computed from it into workspace.
  *   U          optional precomputed adadim_cholesky_inverse_factor of the same H, or NULL.
@@ -142,8 +152,8 @@ ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, float 
  *   workspace  adadim_workspace_bytes(ADADIM_WS_GPTQ, out, in, bits, group), 256-byte aligned.
  */
 ADADIM_API int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
-                         const float* H, const float* U, int bits, int group, int dim,
-                         float percdamp, int blocksize,
+                         const float* H, const double* U, int bits, int group, int dim,
+                         double percdamp, int blocksize,
                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                          double* gptq_loss, int* status_dev,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
@@ -168,7 +178,7 @@ ADADIM_API int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int6
  */
 ADADIM_API int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
                          const float* H, int bits, int group, int dim,
-                         float percdamp, int blocksize,
+                         double percdamp, int blocksize,
                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                          double* gptq_loss, int32_t* perm_out, int* status_dev,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
@@ -205,15 +215,18 @@ ADADIM_API int adadim_score_select(const void* W, int wdtype, int64_t out, int64
  *              ADADIM_STATIC_SCRATCH_BYTES (for example out = in = 1024 fits, out = in = 2048
  *              does not); larger layers are refused with ADADIM_ERR_WORKSPACE and nothing is
  *              launched.
- *   First call The first call on each device looks up the array's device address; make that
- *              first call on a device outside any stream capture.
+ *   First call The first call on each device looks up the array's device address.  With the
+ *              CUDA runtime's lazy loading this lookup is also the moment the 16 MiB become
+ *              resident on that device, so make the first call early - before the process
+ *              commits the device's remaining memory, and outside any stream capture.  If the
+ *              memory cannot be had, that call returns ADADIM_ERR_CUDA.
  *   Sharing    All calls on a device use the same array.  It keeps the previous call's
  *              contents, which no call reads (each call rewrites what it uses).  Two calls
  *              whose kernels can overlap on the GPU - different streams, or different host
  *              threads using different streams - race on it and give wrong results: keep
  *              calls on one device ordered on a single stream, or otherwise serialized.
- *   No cudaMalloc, cudaFree or other allocating call is made.  Arguments, results, status
- *   codes and numerical behaviour are otherwise those of adadim_score_select.
+ *   No cudaMalloc, cudaFree or other allocating call is made.  Arguments (validated by the
+ *   same code), results, status codes and numerical behaviour are those of adadim_score_select.
  */
 #define ADADIM_STATIC_SCRATCH_BYTES (16u << 20)
 ADADIM_API int adadim_score_select_static(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,

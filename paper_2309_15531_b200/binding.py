@@ -53,13 +53,13 @@ def lib():
         L.adadim_quantize_rtn.restype = C.c_int
         L.adadim_quantize_rtn.argtypes = [vp, C.c_int, i64, i64, i64, C.c_int, C.c_int, C.c_int, qp, qp, vp]
         L.adadim_cholesky_inverse_factor.restype = C.c_int
-        L.adadim_cholesky_inverse_factor.argtypes = [vp, i64, C.c_float, vp, vp, vp, sz, vp]
+        L.adadim_cholesky_inverse_factor.argtypes = [vp, i64, C.c_double, vp, vp, vp, sz, vp]
         L.adadim_quantize_gptq.restype = C.c_int
-        L.adadim_quantize_gptq.argtypes = [vp, C.c_int, i64, i64, i64, vp, vp, C.c_int, C.c_int, C.c_int, C.c_float,
+        L.adadim_quantize_gptq.argtypes = [vp, C.c_int, i64, i64, i64, vp, vp, C.c_int, C.c_int, C.c_int, C.c_double,
                                            C.c_int, qp, qp, vp, vp, vp, sz, vp]
         L.adadim_quantize_gptq_reordered.restype = C.c_int
         L.adadim_quantize_gptq_reordered.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, C.c_int,
-                                                     C.c_float, C.c_int, qp, qp, vp, vp, vp, vp, sz, vp]
+                                                     C.c_double, C.c_int, qp, qp, vp, vp, vp, vp, sz, vp]
         L.adadim_score_select.restype = C.c_int
         L.adadim_score_select.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, qp, qp, vp, vp, vp, vp,
                                           sz, vp]
@@ -150,7 +150,7 @@ def quantize_rtn(W: torch.Tensor, bits: int, group: int, dim: int = DIM_BOTH,
 def cholesky_inverse_factor(H: torch.Tensor, percdamp: float = 0.01, status: Optional[torch.Tensor] = None,
                             workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
     n = H.shape[0]
-    U = torch.empty(n, n, dtype=torch.float32, device=H.device)
+    U = torch.empty(n, n, dtype=torch.float64, device=H.device)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_FACTOR, 0, n), H.device)
     rc = lib().adadim_cholesky_inverse_factor(H.data_ptr(), n, percdamp, U.data_ptr(),

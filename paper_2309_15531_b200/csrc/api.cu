@@ -13,11 +13,11 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
                  const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* err, int* chosen, int* status_dev,
                  void* workspace, cudaStream_t st);
 size_t factor_workspace_bytes(int64_t n);
-int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
+int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* status_dev, void* workspace,
                   cudaStream_t st, const int* perm);
 size_t gptq_workspace_bytes(int64_t out, int64_t in);
-int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const float* U,
-                int bits, int group, int dim, float percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const double* U,
+                int bits, int group, int dim, double percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                 double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st, bool reorder, int* perm_out);
 
 namespace {
@@ -45,12 +45,27 @@ int check_qtensor(const adadim_qtensor* q) {
   return ADADIM_OK;
 }
 
-int reset_status(int* status_dev, cudaStream_t st) {
-  if (status_dev != nullptr) ADADIM_CUDA_TRY(cudaMemsetAsync(status_dev, 0, sizeof(int), st));
+}  // namespace
+
+int check_score_args(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, int bits,
+                     int group, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, const double* err,
+                     const int* chosen) {
+  int rc = check_quant_params(bits, group, true);
+  if (rc != ADADIM_OK) return rc;
+  if (out <= 0 || in <= 0) return ADADIM_ERR_SHAPE;
+  rc = check_weight(W, wdtype, out, in, ldw);
+  if (rc != ADADIM_OK) return rc;
+  if (in % 64 != 0 || out % 128 != 0) return ADADIM_ERR_SHAPE;
+  if (q_oc == nullptr && q_ic == nullptr) return ADADIM_ERR_NULL;
+  if (q_oc != nullptr && in % group != 0) return ADADIM_ERR_SHAPE;
+  if (q_ic != nullptr && out % group != 0) return ADADIM_ERR_SHAPE;
+  if (q_oc != nullptr && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
+  if (q_ic != nullptr && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
+  if (H == nullptr || err == nullptr || chosen == nullptr) return ADADIM_ERR_NULL;
+  if (!aligned16(H)) return ADADIM_ERR_ALIGN;
   return ADADIM_OK;
 }
 
-}  // namespace
 }  // namespace adadim
 
 using namespace adadim;
@@ -99,9 +114,8 @@ int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_tokens, int64
   if (in == 0) return ADADIM_OK;
   if (H == nullptr) return ADADIM_ERR_NULL;
   if (!aligned16(H)) return ADADIM_ERR_ALIGN;
-  int rc = reset_status(status_dev, st);
-  if (rc != ADADIM_OK) return rc;
   if (n_tokens == 0) return ADADIM_OK;
+  int rc = ADADIM_OK;
   if (X == nullptr) return ADADIM_ERR_NULL;
   const int64_t esz = xdtype == ADADIM_BF16 ? 2 : 4;
   if (!aligned16(X) || (ldx * esz) % 16 != 0) return ADADIM_ERR_ALIGN;
@@ -131,22 +145,20 @@ int adadim_quantize_rtn(const void* W, int wdtype, int64_t out, int64_t in, int6
   return rtn_launch(W, wdtype, out, in, ldw, bits, group, dim, oc ? *q_oc : none, ic ? *q_ic : none, st);
 }
 
-int adadim_cholesky_inverse_factor(const float* H, int64_t in, float percdamp, float* U, int* status_dev,
+int adadim_cholesky_inverse_factor(const float* H, int64_t in, double percdamp, double* U, int* status_dev,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (in < 0 || in % 64 != 0) return ADADIM_ERR_SHAPE;
-  if (!(percdamp >= 0.0f) || !(percdamp < 1e6f)) return ADADIM_ERR_PARAM;
+  if (!(percdamp >= 0.0) || !(percdamp < 1e6)) return ADADIM_ERR_PARAM;
   if (in == 0) return ADADIM_OK;
   if (H == nullptr || U == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
   if (!aligned16(H) || !aligned16(U) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
   if (workspace_bytes < factor_workspace_bytes(in)) return ADADIM_ERR_WORKSPACE;
-  int rc = reset_status(status_dev, st);
-  if (rc != ADADIM_OK) return rc;
   return factor_launch(H, in, percdamp, U, status_dev, workspace, st, nullptr);
 }
 
 int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H,
-                         const float* U, int bits, int group, int dim, float percdamp, int blocksize,
+                         const double* U, int bits, int group, int dim, double percdamp, int blocksize,
                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* gptq_loss, int* status_dev,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -154,7 +166,7 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
-  if (!(percdamp >= 0.0f) || !(percdamp < 1e6f)) return ADADIM_ERR_PARAM;
+  if (!(percdamp >= 0.0) || !(percdamp < 1e6)) return ADADIM_ERR_PARAM;
   if (out < 0 || in < 0) return ADADIM_ERR_SHAPE;
   if (out == 0 || in == 0) return ADADIM_OK;
   rc = check_weight(W, wdtype, out, in, ldw);
@@ -166,14 +178,12 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
   if (oc && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
   if (ic && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
   if (workspace_bytes < gptq_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
-  rc = reset_status(status_dev, st);
-  if (rc != ADADIM_OK) return rc;
   return gptq_launch(W, wdtype, out, in, ldw, H, U, bits, group, dim, percdamp, q_oc, q_ic, gptq_loss, status_dev,
                      workspace, st, false, nullptr);
 }
 
 int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H,
-                                   int bits, int group, int dim, float percdamp, int blocksize,
+                                   int bits, int group, int dim, double percdamp, int blocksize,
                                    const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* gptq_loss,
                                    int32_t* perm_out, int* status_dev, void* workspace, size_t workspace_bytes,
                                    void* cuda_stream) {
@@ -182,7 +192,7 @@ int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
-  if (!(percdamp >= 0.0f) || !(percdamp < 1e6f)) return ADADIM_ERR_PARAM;
+  if (!(percdamp >= 0.0) || !(percdamp < 1e6)) return ADADIM_ERR_PARAM;
   if (out < 0 || in < 0) return ADADIM_ERR_SHAPE;
   if (out == 0 || in == 0) return ADADIM_OK;
   rc = check_weight(W, wdtype, out, in, ldw);
@@ -194,8 +204,6 @@ int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64
   if (oc && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
   if (ic && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
   if (workspace_bytes < gptq_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
-  rc = reset_status(status_dev, st);
-  if (rc != ADADIM_OK) return rc;
   return gptq_launch(W, wdtype, out, in, ldw, H, nullptr, bits, group, dim, percdamp, q_oc, q_ic, gptq_loss,
                      status_dev, workspace, st, true, perm_out);
 }
@@ -204,22 +212,11 @@ int adadim_score_select(const void* W, int wdtype, int64_t out, int64_t in, int6
                         int group, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* err, int* chosen,
                         int* status_dev, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group, true);
+  const int rc = check_score_args(W, wdtype, out, in, ldw, H, bits, group, q_oc, q_ic, err, chosen);
   if (rc != ADADIM_OK) return rc;
-  if (out <= 0 || in <= 0) return ADADIM_ERR_SHAPE;
-  rc = check_weight(W, wdtype, out, in, ldw);
-  if (rc != ADADIM_OK) return rc;
-  if (in % 64 != 0 || out % 128 != 0) return ADADIM_ERR_SHAPE;
-  if (q_oc == nullptr && q_ic == nullptr) return ADADIM_ERR_NULL;
-  if (q_oc != nullptr && in % group != 0) return ADADIM_ERR_SHAPE;
-  if (q_ic != nullptr && out % group != 0) return ADADIM_ERR_SHAPE;
-  if (q_oc != nullptr && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
-  if (q_ic != nullptr && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
-  if (H == nullptr || err == nullptr || chosen == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
-  if (!aligned16(H) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
+  if (workspace == nullptr) return ADADIM_ERR_NULL;
+  if (!aligned256(workspace)) return ADADIM_ERR_ALIGN;
   if (workspace_bytes < score_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
-  rc = reset_status(status_dev, st);
-  if (rc != ADADIM_OK) return rc;
   return score_launch(W, wdtype, out, in, ldw, H, bits, group, q_oc, q_ic, err, chosen, status_dev, workspace, st);
 }
 

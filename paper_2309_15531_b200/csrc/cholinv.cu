@@ -6,7 +6,7 @@
 // Hd^-1 = (P L^-1 P)^T (P L^-1 P).  This needs one factorization and one triangular inverse
 // instead of a factorization, a full inverse and a second factorization.  All arithmetic is
 // binary64, the large products on the fp64 matrix instruction (the factor decides GPTQ's rounding, so it is kept well inside
-// the fp32 precision of U); U is rounded to fp32 on output.
+// the fp32 precision of U); U is returned in binary64 as well.
 //
 //   factorization : 64-column panels (diagonal block on one CTA, then the panel below it
 //                   multiplied by the inverted diagonal block).  Panels are grouped four at a
@@ -303,7 +303,7 @@ damp_kernel(const float* __restrict__ H, int64_t n, double percdamp, double* sta
     if (threadIdx.x < m) red[threadIdx.x] += red[threadIdx.x + m];
     __syncthreads();
   }
-  if (threadIdx.x == 0) stats[0] = percdamp * red[0] / static_cast<double>(n);
+  if (threadIdx.x == 0) stats[0] = percdamp * (red[0] / static_cast<double>(n));
 }
 
 // A[r][c] = Hd[p(n-1-r)][p(n-1-c)] on and below the diagonal, 0 above it; p is the column order
@@ -726,11 +726,11 @@ merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __rest
 
 // U[i][j] = Linv[n-1-i][n-1-j] for i <= j, else 0
 __global__ void __launch_bounds__(256)
-emit_kernel(const double* __restrict__ A, int64_t n, float* __restrict__ U) {
+emit_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ U) {
   int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
   if (e >= n * n) return;
   int64_t i = e / n, j = e % n;
-  U[e] = i <= j ? static_cast<float>(A[(n - 1 - i) * n + (n - 1 - j)]) : 0.0f;
+  U[e] = i <= j ? A[(n - 1 - i) * n + (n - 1 - j)] : 0.0;
 }
 
 struct FactorLayout { size_t a_off, t_off, dinv_off, stats_off, total; };
@@ -749,7 +749,7 @@ FactorLayout factor_layout(int64_t n) {
 
 size_t factor_workspace_bytes(int64_t n) { return factor_layout(n).total; }
 
-int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
+int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* status_dev, void* workspace,
                   cudaStream_t st, const int* perm) {
   FactorLayout Lo = factor_layout(n);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -764,22 +764,17 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
   // rank update of the next group's own columns) runs on a high-priority stream; the rest of each
   // group's rank update runs beside it on a second stream.  Every kernel of the chain fits on an
   // SM next to one CTA of the rank update, so the chain is scheduled as soon as any CTA retires.
-  cudaStream_t chain = nullptr, side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_panels = nullptr, ev_rest = nullptr, ev_join = nullptr;
-  int prio_least = 0, prio_greatest = 0;
-  ADADIM_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
-  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&chain, cudaStreamNonBlocking, prio_greatest));
-  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, prio_least));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_panels, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_rest, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
+  ForkedStreams fs;                                  // joins and releases on every way out of this function
   bool rest_pending = false;
 
-  damp_kernel<<<1, 256, 0, st>>>(H, n, static_cast<double>(percdamp), stats);
+  damp_kernel<<<1, 256, 0, st>>>(H, n, percdamp, stats);
   build_kernel<<<eb, 256, 0, st>>>(H, n, stats, perm, A);
-  ADADIM_CUDA_TRY(cudaEventRecord(ev_fork, st));
-  ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_fork, 0));
+  {
+    const int rc = fs.open(st);
+    if (rc != ADADIM_OK) return rc;
+  }
+  cudaStream_t chain = fs.chain, side = fs.side;
+  cudaEvent_t ev_panels = fs.ev_a, ev_rest = fs.ev_b;
   for (int g0 = 0; g0 < nb; g0 += kGroup) {
     const int g1 = g0 + kGroup < nb ? g0 + kGroup : nb;
     for (int k = g0; k < g1; ++k) {
@@ -808,16 +803,10 @@ int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* stat
       }
     }
   }
-  if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
-  ADADIM_CUDA_TRY(cudaEventRecord(ev_join, chain));
-  ADADIM_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
-  // destruction is deferred by the runtime until the work already enqueued has finished
-  cudaEventDestroy(ev_fork);
-  cudaEventDestroy(ev_panels);
-  cudaEventDestroy(ev_rest);
-  cudaEventDestroy(ev_join);
-  cudaStreamDestroy(chain);
-  cudaStreamDestroy(side);
+  {
+    const int rc = fs.join();
+    if (rc != ADADIM_OK) return rc;
+  }
   seed_kernel<<<nb, 256, 0, st>>>(A, n, dinv);
   if (n > kNB) {
     const unsigned pairs = static_cast<unsigned>((n + 2 * kNB - 1) / (2 * kNB));

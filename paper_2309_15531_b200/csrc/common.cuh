@@ -23,6 +23,72 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Argument rules shared by adadim_score_select and adadim_score_select_static (everything but
+// the workspace).  Defined in api.cu.
+int check_score_args(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, int bits,
+                     int group, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, const double* err,
+                     const int* chosen);
+
+// The two helper streams of one factor / GPTQ call: a high-priority stream for the chain of small
+// dependent kernels and a low-priority one for the bulk work that runs beside it, plus the events
+// that order them.  open() makes the chain stream wait for everything already enqueued on the
+// caller's stream.  The destructor runs on EVERY exit path, error returns included: it makes the
+// caller's stream wait for whatever was enqueued on both helper streams (so the caller may free
+// or reuse the workspace in stream order as usual) and releases streams and events; the runtime
+// defers their destruction until the enqueued work has finished.
+struct ForkedStreams {
+  cudaStream_t caller = nullptr, chain = nullptr, side = nullptr;
+  cudaEvent_t ev_a = nullptr, ev_b = nullptr, ev_join = nullptr;
+  bool joined = false;
+  int open(cudaStream_t st) {
+    caller = st;
+    int lo = 0, hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaStreamCreateWithPriority(&chain, cudaStreamNonBlocking, hi) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, lo) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&ev_a, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&ev_b, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaEventRecord(ev_join, caller) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (cudaStreamWaitEvent(chain, ev_join, 0) != cudaSuccess) return ADADIM_ERR_CUDA;
+    return ADADIM_OK;
+  }
+  // the caller's stream waits for everything enqueued so far on both helper streams
+  int join() {
+    if (ev_join == nullptr) return ADADIM_ERR_CUDA;
+    bool ok = true;
+    if (side != nullptr) ok = cudaEventRecord(ev_join, side) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
+    if (chain != nullptr) ok = cudaEventRecord(ev_join, chain) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
+    joined = true;
+    return ok ? ADADIM_OK : ADADIM_ERR_CUDA;
+  }
+  ~ForkedStreams() {
+    if (!joined && ev_join != nullptr) join();
+    if (ev_a != nullptr) cudaEventDestroy(ev_a);
+    if (ev_b != nullptr) cudaEventDestroy(ev_b);
+    if (ev_join != nullptr) cudaEventDestroy(ev_join);
+    if (chain != nullptr) cudaStreamDestroy(chain);
+    if (side != nullptr) cudaStreamDestroy(side);
+  }
+  ForkedStreams() = default;
+  ForkedStreams(const ForkedStreams&) = delete;
+  ForkedStreams& operator=(const ForkedStreams&) = delete;
+};
+
+// Layout of GPTQ's binary64 working weights (internal to one call's workspace): tiles of 32 rows
+// x 16 columns, 4 KB each and contiguous, tile (R, C) at ((R * (in / 16)) + C) * 512 doubles.
+// Inside a tile row r keeps its eight 16-byte column pairs at pair position p ^ (r & 7).  A tile
+// is what one warp of the trailing update adds in one bulk operation and what the block kernel
+// fetches in one bulk copy; the pair swizzle lets 32 threads that each own a row touch a tile
+// without shared-memory bank conflicts.
+constexpr int kWcTileRows = 32, kWcTileCols = 16, kWcTileElems = 512;
+__host__ __device__ __forceinline__ int wc_in_tile(int r, int c) {          // r < 32, c < 16
+  return r * 16 + ((((c >> 1) ^ (r & 7)) << 1) | (c & 1));
+}
+__host__ __device__ __forceinline__ int64_t wc_index(int64_t row, int64_t col, int64_t in) {
+  return ((row >> 5) * (in >> 4) + (col >> 4)) * kWcTileElems + wc_in_tile(static_cast<int>(row & 31), static_cast<int>(col & 15));
+}
+
 // Record a device-side condition: the first error wins.
 __device__ __forceinline__ void report(int* status_dev, int code) {
   if (status_dev != nullptr) atomicCAS(status_dev, ADADIM_OK, code);

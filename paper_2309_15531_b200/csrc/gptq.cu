@@ -7,40 +7,55 @@
 //                     columns being worked on live in registers.
 //   trailing update - W[:, after the block] -= Err[out,128] * U[block rows, after the block]
 //                     on the tensor cores with exactly sliced bf16 operands (gptq_tc.cu).
+// The working weights, the factor and every update inside a block are binary64: a weight is
+// rounded thousands of columns after the first error was folded into it, and a binary32 copy
+// re-rounded at every update drifts far enough (a few 1e-6 of a quantization step) to move
+// individual rounding decisions, each of which then changes everything after it.  Only the
+// decision itself (group parameters and the code of the weight as it stands, rounded once to
+// binary32) is binary32 arithmetic, as the quantizer's definition says.
 // Rows are independent under per-OC grouping; under per-IC grouping a group couples g
 // consecutive rows of one column, which is why a CTA owns a whole 128-row slab.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include "common.cuh"
+#include "umma.cuh"
 
 namespace adadim {
 
 struct TrailPlan {
-  CUtensorMap e[3], u[3], w;
-  float* Wc;
+  CUtensorMap e[3], u[3];
+  double* Wc;
   int64_t rows_total, in;
   int sm_count;
 };
-int trail_split_u(const float* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st);
-int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
+int trail_split_u(const double* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st);
+int trail_plan(TrailPlan* plan, double* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
                const __nv_bfloat16* const u[3]);
 int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int tiles_per_cta, int* status_dev, cudaStream_t st);
 
 size_t factor_workspace_bytes(int64_t n);
-int factor_launch(const float* H, int64_t n, float percdamp, float* U, int* status_dev, void* workspace,
+int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* status_dev, void* workspace,
                   cudaStream_t st, const int* perm);
 
 namespace {
 
 constexpr int kBlk = 128;            // lazy-batch block width (columns) and slab height (rows)
 constexpr int kSub = 32;             // columns held in registers at a time
-constexpr int kPad = kBlk + 1;       // shared-memory row pitch (floats): conflict-free column access
+constexpr int kLater = kBlk - kSub;  // columns of a block that are not in registers during its first sub-block
+constexpr int kEP = kSub + 1;        // row pitch (doubles) of the current sub-block's errors
+constexpr int kLaterTiles = (kBlk / kWcTileRows) * (kLater / kWcTileCols);       // 24 tiles of the working-weight layout
+constexpr int kFirstTiles = (kBlk / kWcTileRows) * (kSub / kWcTileCols);         // 8 tiles
+
+// The U block is upper triangular: row tile t (rows 32 t .. 32 t + 31) keeps columns 32 t .. 127
+// only, with row pitch 128 - 32 t.
+__host__ __device__ constexpr int u_tile_off(int t) { return 32 * (128 * t - 16 * t * (t - 1)); }
+__host__ __device__ constexpr int u_tile_pitch(int t) { return kBlk - 32 * t; }
+constexpr int kUPacked = u_tile_off(4);              // 10240 doubles
 
 template <typename T>
 __global__ void __launch_bounds__(256)
 init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const float* __restrict__ H, int ndim,
-            float* __restrict__ Wc) {
+            double* __restrict__ Wc) {
   int64_t e = (static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x) * 8;
   if (e >= out * in) return;
   int64_t o = e / in, i = e % in;
@@ -50,15 +65,18 @@ init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const
   for (int k = 0; k < 8; ++k)
     if (H[(i + k) * in + (i + k)] == 0.0f) v[k] = 0.0f;        // dead column
   for (int d = 0; d < ndim; ++d) {
-    float4* dst = reinterpret_cast<float4*>(Wc + static_cast<int64_t>(d) * out * in + e);
-    dst[0] = make_float4(v[0], v[1], v[2], v[3]);
-    dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+    double* dst = Wc + static_cast<int64_t>(d) * out * in;
+#pragma unroll
+    for (int k = 0; k < 4; ++k)          // four column pairs of one row of one tile
+      *reinterpret_cast<double2*>(dst + wc_index(o, i + 2 * k, in)) =
+          make_double2(static_cast<double>(v[2 * k]), static_cast<double>(v[2 * k + 1]));
   }
 }
 
 struct BlockArgs {
-  float* Wc;                 // [ndim][out][in] working weights
-  const float* U;            // [in][in]
+  double* Wc;                // [ndim] working weights of [out][in] each, in the tiled layout of wc_index()
+  const double* U;           // [in][in]
+  int* status_dev;
   __nv_bfloat16* Ep[3];      // [ndim*out][128] errors as three fixed-point bf16 pieces
   double* loss_part;         // [ndim][out/128]
   adadim_qtensor q[2];       // outputs for the dimension(s) in flight
@@ -99,17 +117,17 @@ order_kernel(const float* __restrict__ H, int64_t n, int* __restrict__ perm, int
   if (i < n) { rank[i] = before; perm[before] = static_cast<int>(i); }
 }
 
-// Working copies in the quantization order: Wc[d][o][i] = W[o][perm[i]] (0 for dead columns).
+// Working copies in the quantization order: element (o, i) of copy d = W[o][perm[i]] (0 for dead columns).
 template <typename T>
 __global__ void __launch_bounds__(256)
 init_perm_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const float* __restrict__ H,
-                 const int* __restrict__ perm, int ndim, float* __restrict__ Wc) {
+                 const int* __restrict__ perm, int ndim, double* __restrict__ Wc) {
   const int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
   if (e >= out * in) return;
   const int64_t o = e / in, c = perm[e % in];
   float v = static_cast<float>(W[o * ldw + c]);
   if (H[c * in + c] == 0.0f) v = 0.0f;
-  for (int d = 0; d < ndim; ++d) Wc[static_cast<int64_t>(d) * out * in + e] = v;
+  for (int d = 0; d < ndim; ++d) Wc[static_cast<int64_t>(d) * out * in + wc_index(o, e % in, in)] = static_cast<double>(v);
 }
 
 // Static per-OC groups: parameters of every group of g consecutive original columns, from the
@@ -177,40 +195,60 @@ __device__ __forceinline__ int ordered_key(float v) {
 }
 __device__ __forceinline__ float from_ordered_key(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7fffffff)); }
 
+// Position (in doubles) of element (r, lc) of the slab's later columns in shared memory: the 24
+// tiles are kept as fetched, tile (r / 32, lc / 16) at slot (r / 32) * 6 + lc / 16.
+__device__ __forceinline__ int later_at(int r, int lc) {
+  return ((r >> 5) * (kLater / kWcTileCols) + (lc >> 4)) * kWcTileElems + wc_in_tile(r & 31, lc & 15);
+}
+
 // W[:, later columns] -= Err[:, this sub-block] * U[sub-block rows, later columns] for the whole
-// 128-row slab in shared memory.  A row-per-thread loop needs one warp-uniform U value per
-// multiply-add, all of it through the shared-memory return path, which bounds it at a quarter of
-// the multiply-add rate; here a thread owns 8 rows x CW columns, so 8 + CW loads feed 8 CW
-// multiply-adds.  Every element still receives its 32 updates in the same order as before.
-template <int CW>
-__device__ __forceinline__ void lazy_update(float* __restrict__ Ws, const float* __restrict__ Us,
-                                            const float* __restrict__ Es, int cbase, int tid) {
+// 128-row slab in shared memory, in binary64.  A row-per-thread loop needs one warp-uniform U
+// value per multiply-add, all of it through the shared-memory return path; here a thread owns
+// 8 rows x CH columns at a time (two such column pieces), so 8 + CH loads feed 8 CH
+// multiply-adds.  Every element receives its 32 updates in column order.
+//   Wt  later columns of the slab (tiles, see later_at)
+//   Ut  row tile of the packed U block that holds the sub-block's rows (pitch up)
+//   Es  the sub-block's errors, Es[r * kEP + ii]
+template <int CH>
+__device__ __forceinline__ void lazy_update(double* __restrict__ Wt, const double* __restrict__ Ut, int up,
+                                            const double* __restrict__ Es, int cbase, int tid) {
   const int r0 = (tid >> 3) * 8;
-  const int col0 = cbase + kSub + (tid & 7) * CW;
-  float acc[8][CW];
+#pragma unroll 1
+  for (int piece = 0; piece < 2; ++piece) {
+    const int lc = ((tid & 7) * 2 + piece) * CH;     // first of this thread's columns among the later ones (even)
+    double acc[8][CH];
+    int at[CH / 2];                                  // position of row r0's column pairs; row r0 + m differs by a swizzle
 #pragma unroll
-  for (int m = 0; m < 8; ++m)
+    for (int n2 = 0; n2 < CH / 2; ++n2) at[n2] = later_at(r0, cbase + lc + 2 * n2);
 #pragma unroll
-    for (int n = 0; n < CW; ++n) acc[m][n] = Ws[(r0 + m) * kPad + col0 + n];
-#pragma unroll 4
-  for (int ii = 0; ii < kSub; ++ii) {
-    float e[8], u[CW];
+    for (int m = 0; m < 8; ++m)
 #pragma unroll
-    for (int m = 0; m < 8; ++m) e[m] = Es[(r0 + m) * kPad + cbase + ii];
+      for (int n2 = 0; n2 < CH / 2; ++n2) {
+        // r0 is a multiple of 8, so row r0 + m has swizzle m: pair position p ^ m, 16 doubles further per row
+        const double2 t = *reinterpret_cast<const double2*>(Wt + (at[n2] ^ (m << 1)) + m * 16);
+        acc[m][2 * n2] = t.x; acc[m][2 * n2 + 1] = t.y;
+      }
+#pragma unroll 2
+    for (int ii = 0; ii < kSub; ++ii) {
+      double e[8], u[CH];
 #pragma unroll
-    for (int n4 = 0; n4 < CW / 4; ++n4) {
-      const float4 t = *reinterpret_cast<const float4*>(Us + (cbase + ii) * kBlk + col0 + 4 * n4);
-      u[4 * n4] = t.x; u[4 * n4 + 1] = t.y; u[4 * n4 + 2] = t.z; u[4 * n4 + 3] = t.w;
+      for (int m = 0; m < 8; ++m) e[m] = Es[(r0 + m) * kEP + ii];
+#pragma unroll
+      for (int n2 = 0; n2 < CH / 2; ++n2) {
+        const double2 t = *reinterpret_cast<const double2*>(Ut + ii * up + kSub + lc + 2 * n2);
+        u[2 * n2] = t.x; u[2 * n2 + 1] = t.y;
+      }
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+#pragma unroll
+        for (int n = 0; n < CH; ++n) acc[m][n] = fma(-e[m], u[n], acc[m][n]);
     }
 #pragma unroll
     for (int m = 0; m < 8; ++m)
 #pragma unroll
-      for (int n = 0; n < CW; ++n) acc[m][n] = fmaf(-e[m], u[n], acc[m][n]);
+      for (int n2 = 0; n2 < CH / 2; ++n2)
+        *reinterpret_cast<double2*>(Wt + (at[n2] ^ (m << 1)) + m * 16) = make_double2(acc[m][2 * n2], acc[m][2 * n2 + 1]);
   }
-#pragma unroll
-  for (int m = 0; m < 8; ++m)
-#pragma unroll
-    for (int n = 0; n < CW; ++n) Ws[(r0 + m) * kPad + col0 + n] = acc[m][n];
 }
 
 template <int BITS, int G>
@@ -219,14 +257,18 @@ block_kernel(const BlockArgs a) {
   constexpr float maxq = static_cast<float>((1 << BITS) - 1);
   constexpr float rcp_maxq = 1.0f / maxq;            // correctly rounded at compile time
   constexpr int NG = kBlk / G;                       // per-IC groups in the slab
-  extern __shared__ float sm[];
-  float* Ws = sm;                                    // [128][129] slab of the working weights
-  float* Us = Ws + kBlk * kPad;                      // [128][128] block of U (upper triangle used)
-  float* Es = Us + kBlk * kBlk;                      // [128][129] errors
-  float* invd = Es + kBlk * kPad;                    // [128] 1 / U[i,i]
-  float* red = invd + kBlk;                          // [2][4][2] per-IC min / max exchange
+  extern __shared__ __align__(128) double smd[];
+  double* Wt = smd;                                  // 24 tiles: columns 32..127 of the slab (later_at)
+  double* Us = Wt + kLaterTiles * kWcTileElems;      // packed upper block-triangle of the U block
+  double* Es = Us + kUPacked;                        // [128][33] errors of the current sub-block; first the
+                                                     // landing zone of the 8 tiles of columns 0..31
+  double* invd = Es + kBlk * kEP;                    // [128] 1 / U[i,i]
+  float* gridr = reinterpret_cast<float*>(invd + kBlk);   // [128] slicing grid of every row's errors
+  float* red = gridr + kBlk;                         // [2][4][2] per-IC min / max exchange
   uint16_t* Ss = reinterpret_cast<uint16_t*>(red + 16);   // [NG][128] per-IC scales (fp16 bits)
   uint16_t* Zs = Ss + NG * kBlk;                          // [NG][128]
+  __shared__ uint64_t bar[2];
+  __shared__ int dead_flag;
 
   const int d = blockIdx.y;
   const bool is_ic = a.dim_of[d] == ADADIM_DIM_IC;
@@ -234,58 +276,85 @@ block_kernel(const BlockArgs a) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kBlk;
   const int64_t row = row0 + tid;
-  float* Wd = a.Wc + static_cast<int64_t>(d) * a.out * a.in;
+  const double* Wd = a.Wc + static_cast<int64_t>(d) * a.out * a.in;
 
-  // Stage the U block and the slab (coalesced), then work row-per-thread; eight rows' worth of
-  // loads are in flight before the first is stored, so each copy costs 4 memory latencies, not 32.
-  // The kernel may have been scheduled while the launch before it in the stream (the update of this
-  // block's columns) is still finishing: U does not depend on it and is staged first; everything
-  // after the wait sees that launch's results.
-#pragma unroll 1
-  for (int e0 = 0; e0 < kBlk * kBlk / 4; e0 += 8 * kBlk) {
-    float4 uv[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
-      uv[u] = *reinterpret_cast<const float4*>(a.U + static_cast<int64_t>(a.i1 + r) * a.in + a.i1 + c4);
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
-      *reinterpret_cast<float4*>(Us + r * kBlk + c4) = uv[u];
-    }
+  // Staging by bulk copies: one memory latency for the U block and one for the slab.  The kernel
+  // may have been scheduled while the launch before it in the stream (the update of this block's
+  // columns) is still finishing: U does not depend on it and is fetched first; everything after
+  // the wait sees that launch's results.
+  if (tid == 0) {
+    ptx::mbar_init(&bar[0], 1);
+    ptx::mbar_init(&bar[1], 1);
+    dead_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::mbar_arrive_expect_tx(&bar[0], kUPacked * sizeof(double));
+    ptx::mbar_arrive_expect_tx(&bar[1], (kLaterTiles + kFirstTiles) * kWcTileElems * sizeof(double));
+  }
+  __syncthreads();
+  {
+    // row tid of the U block: columns from the start of its 32-row tile to the end of the block
+    const int t = tid >> 5, up = u_tile_pitch(t);
+    ptx::bulk_load(Us + u_tile_off(t) + (tid & 31) * up, a.U + static_cast<int64_t>(a.i1 + tid) * a.in + a.i1 + 32 * t,
+                   static_cast<uint32_t>(up * sizeof(double)), &bar[0]);
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
-#pragma unroll 1
-  for (int e0 = 0; e0 < kBlk * kBlk / 4; e0 += 8 * kBlk) {
-    float4 wv[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
-      wv[u] = *reinterpret_cast<const float4*>(Wd + (row0 + r) * a.in + a.i1 + c4);
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int e = e0 + u * kBlk + tid, r = e >> 5, c4 = (e & 31) * 4;
-      Ws[r * kPad + c4 + 0] = wv[u].x; Ws[r * kPad + c4 + 1] = wv[u].y; Ws[r * kPad + c4 + 2] = wv[u].z; Ws[r * kPad + c4 + 3] = wv[u].w;
-    }
+  if (tid < kLaterTiles + kFirstTiles) {
+    // tile tid of the slab: 4 tile rows x 8 tile columns; the first two tile columns land in Es
+    const int tr = tid >> 3, tc = tid & 7;
+    const double* src = Wd + ((row0 / kWcTileRows + tr) * (a.in / kWcTileCols) + a.i1 / kWcTileCols + tc) * kWcTileElems;
+    double* dst = tc < 2 ? Es + (tr * 2 + tc) * kWcTileElems : Wt + (tr * (kLater / kWcTileCols) + tc - 2) * kWcTileElems;
+    ptx::bulk_load(dst, src, kWcTileElems * sizeof(double), &bar[1]);
   }
-  __syncthreads();
-  invd[tid] = 1.0f / Us[tid * kBlk + tid];
-  __syncthreads();
+  const bool staged = ptx::mbar_wait(&bar[0], 0, &dead_flag, a.status_dev) &
+                      ptx::mbar_wait(&bar[1], 0, &dead_flag, a.status_dev);
+  if (!__syncthreads_and(staged)) {
+    // a copy did not arrive in time (reported as ADADIM_ERR_TIMEOUT): give what is in flight one more
+    // bounded wait so that nothing lands in shared memory after the CTA has gone, then stop
+    const long long c0 = clock64();
+    while (!(ptx::mbar_try_wait(&bar[0], 0) && ptx::mbar_try_wait(&bar[1], 0)) && clock64() - c0 < ptx::kWaitLimit) {}
+    return;
+  }
+  invd[tid] = 1.0 / Us[u_tile_off(tid >> 5) + (tid & 31) * u_tile_pitch(tid >> 5) + (tid & 31)];
 
-  float* wrow = Ws + tid * kPad;
-  float* erow = Es + tid * kPad;
+  double* erow = Es + tid * kEP;
   GroupParams gp = {1.0f, 0.0f, 0.0f};
   double loss = 0.0;
+  float emax = 0.0f;
 
 #pragma unroll 1
   for (int sb = 0; sb < kBlk / kSub; ++sb) {
     const int cbase = sb * kSub;
-    float w[kSub], err[kSub];
+    const int up = u_tile_pitch(sb);
+    const double* Ut = Us + u_tile_off(sb);
+    double w[kSub];
     uint32_t cw[BITS] = {};
+    if (sb == 0) {
+      // this row's first 32 weights from the landing zone, which then becomes the error array
 #pragma unroll
-    for (int k = 0; k < kSub; ++k) w[k] = wrow[cbase + k];
+      for (int k2 = 0; k2 < kSub / 2; ++k2) {
+        const double2 t = *reinterpret_cast<const double2*>(
+            Es + ((tid >> 5) * 2 + (k2 >> 3)) * kWcTileElems + wc_in_tile(lane, 2 * (k2 & 7)));
+        w[2 * k2] = t.x; w[2 * k2 + 1] = t.y;
+      }
+      __syncthreads();                               // every row has been read before the first error is written
+    } else {
+      // columns cbase .. cbase + 31 are later columns cbase - 32 ..; their slots are free from here
+      // on and take the previous sub-block's errors, rounded to binary32, for the slicing at the end:
+      // errors of sub-block j at later columns 32 j .. 32 j + 15 (two floats per slot)
+      float4 ef[kSub / 4];
+#pragma unroll
+      for (int k = 0; k < kSub / 4; ++k)
+        ef[k] = make_float4(static_cast<float>(erow[4 * k]), static_cast<float>(erow[4 * k + 1]),
+                            static_cast<float>(erow[4 * k + 2]), static_cast<float>(erow[4 * k + 3]));
+#pragma unroll
+      for (int k2 = 0; k2 < kSub / 2; ++k2) {
+        const double2 t = *reinterpret_cast<const double2*>(Wt + later_at(tid, cbase - kSub + 2 * k2));
+        w[2 * k2] = t.x; w[2 * k2 + 1] = t.y;
+      }
+#pragma unroll
+      for (int k = 0; k < kSub / 4; ++k)
+        *reinterpret_cast<float4*>(Wt + later_at(tid, cbase - kSub + 2 * k)) = ef[k];
+    }
     uint2 srec[kSub];                                // static per-OC records of these 32 columns
     if (!is_ic && a.static_rec != nullptr) {
 #pragma unroll
@@ -296,6 +365,7 @@ block_kernel(const BlockArgs a) {
 #pragma unroll
     for (int ii = 0; ii < kSub; ++ii) {
       const int i = cbase + ii;                      // column inside the block
+      const float w32 = static_cast<float>(w[ii]);   // the weight as it stands, rounded once: what is quantized
       if (!is_ic && a.static_rec != nullptr) {       // per-OC, static groups: parameters fixed beforehand
         const uint2 rec = srec[ii];
         gp.rcp = __uint_as_float(rec.x);
@@ -303,12 +373,15 @@ block_kernel(const BlockArgs a) {
         gp.z = __half2float(__ushort_as_half(static_cast<unsigned short>(rec.y >> 16)));
       } else if (!is_ic) {
         if ((ii % G) == 0 && (cbase % G) == 0) {     // per-OC: parameters at the group's first column
-          float mn = w[ii], mx = w[ii];
-          if (G == kSub) {
+          float mn = w32, mx = w32;
 #pragma unroll
-            for (int k = 1; k < kSub; ++k) { mn = fminf(mn, w[k]); mx = fmaxf(mx, w[k]); }
-          } else {
-            for (int k = 1; k < G; ++k) { float v = wrow[i + k]; mn = fminf(mn, v); mx = fmaxf(mx, v); }
+          for (int k = 1; k < (G < kSub ? G : kSub); ++k) {
+            const float v = static_cast<float>(w[ii + k < kSub ? ii + k : kSub - 1]);
+            mn = fminf(mn, v); mx = fmaxf(mx, v);
+          }
+          for (int k = kSub; k < G; ++k) {           // the group's columns beyond the ones in registers
+            const float v = static_cast<float>(Wt[later_at(tid, cbase + k - kSub)]);
+            mn = fminf(mn, v); mx = fmaxf(mx, v);
           }
           gp = group_params(mn, mx, maxq, rcp_maxq);
           int64_t idx = row * (a.in / G) + (a.i1 + i) / G;
@@ -318,7 +391,7 @@ block_kernel(const BlockArgs a) {
       } else {                                       // per-IC: parameters of this column's g-row groups
         // warp minimum and maximum in one reduction instruction each, on a key that orders
         // floats as signed integers (negative values have their magnitude bits flipped)
-        const int key = ordered_key(w[ii]);
+        const int key = ordered_key(w32);
         float mn = from_ordered_key(__reduce_min_sync(0xffffffffu, key));
         float mx = from_ordered_key(__reduce_max_sync(0xffffffffu, key));
         if (G > 32) {
@@ -337,20 +410,20 @@ block_kernel(const BlockArgs a) {
           Zs[(tid / G) * kBlk + i] = __half_as_ushort(__float2half_rn(gp.z));
         }
       }
-      const int c = code_of(quotient(w[ii], gp.s, gp.rcp), gp.z, maxq);
+      const int c = code_of(quotient(w32, gp.s, gp.rcp), gp.z, maxq);
       const float qv = __fmul_rn(gp.s, static_cast<float>(c) - gp.z);
-      const float e = (w[ii] - qv) * invd[i];
-      err[ii] = e;
-      erow[i] = e;
-      loss += static_cast<double>(e) * static_cast<double>(e);
+      const double e = (w[ii] - static_cast<double>(qv)) * invd[i];
+      erow[ii] = e;
+      emax = fmaxf(emax, fabsf(static_cast<float>(e)));
+      loss = fma(e, e, loss);
       {
         const int bit = ii * BITS, wi = bit >> 5, sh = bit & 31;
         cw[wi] |= static_cast<uint32_t>(c) << sh;
         if (sh + BITS > 32) cw[wi + 1] |= static_cast<uint32_t>(c) >> (32 - sh);
       }
-      const float* urow = Us + i * kBlk + cbase;
+      const double* urow = Ut + ii * up;
 #pragma unroll
-      for (int jj = ii + 1; jj < kSub; ++jj) w[jj] = fmaf(-e, urow[jj], w[jj]);
+      for (int jj = ii + 1; jj < kSub; ++jj) w[jj] = fma(-e, urow[jj], w[jj]);
     }
     // codes of these 32 columns: BITS whole words of this row's bitstream
     uint32_t* cdst = a.codes[d] + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
@@ -359,30 +432,34 @@ block_kernel(const BlockArgs a) {
     // lazy update of the block's later columns with this sub-block's 32 errors, as a small
     // register-tiled product over the whole slab (see lazy_update)
     __syncthreads();
-    const int later = kBlk - cbase - kSub;
-    if (later == 96) lazy_update<12>(Ws, Us, Es, cbase, tid);
-    else if (later == 64) lazy_update<8>(Ws, Us, Es, cbase, tid);
-    else if (later == 32) lazy_update<4>(Ws, Us, Es, cbase, tid);
+    if (sb == 0) lazy_update<6>(Wt, Ut, up, Es, cbase, tid);
+    else if (sb == 1) lazy_update<4>(Wt, Ut, up, Es, cbase, tid);
+    else if (sb == 2) lazy_update<2>(Wt, Ut, up, Es, cbase, tid);
     __syncthreads();
   }
 
   // ---- outputs: errors (coalesced), per-IC parameters, loss ------------------------------
-  __syncthreads();
-  // errors as three fixed-point bf16 pieces on one grid per row (see gptq_tc.cu)
+  // errors as three fixed-point bf16 pieces on one grid per row (see gptq_tc.cu).  The binary32
+  // errors of sub-blocks 0..2 already sit in the slab's free slots; those of the last one follow.
+#pragma unroll
+  for (int k = 0; k < kSub / 4; ++k)
+    *reinterpret_cast<float4*>(Wt + later_at(tid, kLater - kSub / 2 + 2 * k)) =
+        make_float4(static_cast<float>(erow[4 * k]), static_cast<float>(erow[4 * k + 1]),
+                    static_cast<float>(erow[4 * k + 2]), static_cast<float>(erow[4 * k + 3]));
   {
-    float m = 0.0f;
-    for (int k = 0; k < kBlk; ++k) m = fmaxf(m, fabsf(erow[k]));
-    int ex = (__float_as_int(m) >> 23) & 0xFF;
+    int ex = (__float_as_int(emax) >> 23) & 0xFF;
     ex = ex < 32 ? 32 : (ex > 250 ? 250 : ex);
-    invd[tid] = __int_as_float((ex - 7) << 23);     // grid of this row (invd is free now)
+    gridr[tid] = __int_as_float((ex - 7) << 23);     // grid of this row
   }
   __syncthreads();
   const int64_t ebase = (static_cast<int64_t>(d) * a.out + row0) * kBlk;
-  // thread tid takes column tid of every row r (e = 128 r + tid): a warp stores 64 contiguous bytes
+  // thread tid takes column tid of every row r (e = 128 r + tid): a warp stores 64 contiguous bytes.
+  // Column tid = 32 j + k: float k of the 16 slots that hold sub-block j's errors.
+  const int eslot = (warp < 3 ? kSub * warp : kLater - kSub / 2) + (lane >> 1);
 #pragma unroll 8
   for (int r = 0; r < kBlk; ++r) {
-    const float v = Es[r * kPad + tid];
-    const float g = invd[r];
+    const float v = reinterpret_cast<const float*>(Wt + later_at(r, eslot))[lane & 1];
+    const float g = gridr[r];
     const float inv = __int_as_float(0x7F000000 - __float_as_int(g));   // 1 / g for a power of two, exact
     const float a0 = rintf(v * inv);
     const float r1 = fmaf(-a0, g, v);
@@ -421,7 +498,8 @@ __global__ void loss_kernel(const double* __restrict__ part, int ndim, int slabs
 }
 
 constexpr size_t block_smem_bytes() {
-  return (kBlk * kPad * 2 + kBlk * kBlk + kBlk + 16) * sizeof(float) + 2 * 4 * kBlk * sizeof(uint16_t);
+  return (kLaterTiles * kWcTileElems + kUPacked + kBlk * kEP + kBlk) * sizeof(double) + (kBlk + 16) * sizeof(float) +
+         2 * 4 * kBlk * sizeof(uint16_t);
 }
 
 template <int BITS, int G>
@@ -451,13 +529,13 @@ struct GptqLayout {
 GptqLayout gptq_layout(int64_t out, int64_t in) {
   GptqLayout L;
   size_t off = 0;
-  L.wc_off = off;     off += round_up(static_cast<size_t>(2) * out * in * 4, 256);
+  L.wc_off = off;     off += round_up(static_cast<size_t>(2) * out * in * 8, 256);
   L.err_piece = round_up(static_cast<size_t>(2) * 2 * out * kBlk * 2, 1024);      // two alternating sets
   L.err_off = off;    off += 3 * L.err_piece;
   L.up_piece = round_up(static_cast<size_t>(in) * in * 2, 1024);
   L.up_off = off;     off += 3 * L.up_piece;
   L.loss_off = off;   off += round_up(static_cast<size_t>(2) * (out / kBlk + 1) * 8, 256);
-  L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 4, 256);
+  L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 8, 256);
   L.factor_off = off; off += factor_workspace_bytes(in);
   L.perm_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
   L.rank_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
@@ -468,17 +546,25 @@ GptqLayout gptq_layout(int64_t out, int64_t in) {
   return L;
 }
 
+template <int BITS>
+int block_launch_g(const BlockArgs& a, int group, int slabs, int ndim, cudaStream_t st) {
+  return group == 128 ? block_launch<BITS, 128>(a, slabs, ndim, st)
+       : group == 64  ? block_launch<BITS, 64>(a, slabs, ndim, st)
+                      : block_launch<BITS, 32>(a, slabs, ndim, st);
+}
+
 }  // namespace
 
 size_t gptq_workspace_bytes(int64_t out, int64_t in) { return gptq_layout(out, in).total; }
 
-int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const float* U_in,
-                int bits, int group, int dim, float percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
+int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const double* U_in,
+                int bits, int group, int dim, double percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                 double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st, bool reorder, int* perm_out) {
   GptqLayout L = gptq_layout(out, in);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   BlockArgs a = {};
-  a.Wc = reinterpret_cast<float*>(ws + L.wc_off);
+  a.Wc = reinterpret_cast<double*>(ws + L.wc_off);
+  a.status_dev = status_dev;
   const __nv_bfloat16* ep[3];
   const __nv_bfloat16* up[3];
   for (int k = 0; k < 3; ++k) {
@@ -518,9 +604,9 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
     }
   }
 
-  const float* U = U_in;
+  const double* U = U_in;
   if (U == nullptr || reorder) {                     // a caller's factor belongs to the natural order
-    float* Uw = reinterpret_cast<float*>(ws + L.u_off);
+    double* Uw = reinterpret_cast<double*>(ws + L.u_off);
     int rc = factor_launch(H, in, percdamp, Uw, status_dev, ws + L.factor_off, st, perm);
     if (rc != ADADIM_OK) return rc;
     U = Uw;
@@ -550,67 +636,47 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
   // beside the next block kernel on a second stream, on the SMs the block kernel leaves free.  The
   // error pieces alternate between two sets, so a block kernel never overwrites what the other
   // stream still reads.
-  cudaStream_t chain = nullptr, side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_block = nullptr, ev_rest = nullptr, ev_join = nullptr;
-  int prio_least = 0, prio_greatest = 0;
-  ADADIM_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
-  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&chain, cudaStreamNonBlocking, prio_greatest));
-  ADADIM_CUDA_TRY(cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, prio_least));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_block, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_rest, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
-  ADADIM_CUDA_TRY(cudaEventRecord(ev_fork, st));
-  ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_fork, 0));
-  const int64_t rows_total = static_cast<int64_t>(ndim) * out;
-  // the side-stream launches get the SMs that the block kernel leaves free (finer CTAs were
-  // measured slower: every CTA reloads its 96 KB of error pieces and refills the pipeline)
-  const int free_sms = plan.sm_count - slabs * ndim;
-  const int64_t mblocks = rows_total / kBlk;
-  const int rest_split = free_sms >= mblocks ? static_cast<int>(free_sms / mblocks) : 1;
-  __nv_bfloat16* ep_base[3] = {a.Ep[0], a.Ep[1], a.Ep[2]};
-  bool rest_pending = false;
-  for (int i1 = 0; i1 < in; i1 += kBlk) {
-    a.i1 = i1;
-    for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows_total * kBlk;
-    int rc;
-    if (bits == 3) {
-      rc = group == 128 ? block_launch<3, 128>(a, slabs, ndim, chain) : group == 64 ? block_launch<3, 64>(a, slabs, ndim, chain)
-                                                                                    : block_launch<3, 32>(a, slabs, ndim, chain);
-    } else {
-      rc = group == 128 ? block_launch<4, 128>(a, slabs, ndim, chain) : group == 64 ? block_launch<4, 64>(a, slabs, ndim, chain)
-                                                                                    : block_launch<4, 32>(a, slabs, ndim, chain);
-    }
-    if (rc != ADADIM_OK) return rc;
-    const int tiles_after = static_cast<int>((in - i1 - kBlk) / kBlk);
-    if (tiles_after > 0) {
-      if (tiles_after > 1) ADADIM_CUDA_TRY(cudaEventRecord(ev_block, chain));
-      // the next block's columns were last written by the previous block's side-stream launch
-      if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
-      rest_pending = false;
-      rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, 1, status_dev, chain);
+  {
+    ForkedStreams fs;                                // joins and releases on every way out of this scope
+    rc0 = fs.open(st);
+    if (rc0 != ADADIM_OK) return rc0;
+    cudaStream_t chain = fs.chain, side = fs.side;
+    cudaEvent_t ev_block = fs.ev_a, ev_rest = fs.ev_b;
+    const int64_t rows_total = static_cast<int64_t>(ndim) * out;
+    // the side-stream launches get the SMs that the block kernel leaves free (finer CTAs were
+    // measured slower: every CTA reloads its 96 KB of error pieces and refills the pipeline)
+    const int free_sms = plan.sm_count - slabs * ndim;
+    const int64_t mblocks = rows_total / kBlk;
+    const int rest_split = free_sms >= mblocks ? static_cast<int>(free_sms / mblocks) : 1;
+    __nv_bfloat16* ep_base[3] = {a.Ep[0], a.Ep[1], a.Ep[2]};
+    bool rest_pending = false;
+    for (int i1 = 0; i1 < in; i1 += kBlk) {
+      a.i1 = i1;
+      for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows_total * kBlk;
+      int rc = bits == 3 ? block_launch_g<3>(a, group, slabs, ndim, chain) : block_launch_g<4>(a, group, slabs, ndim, chain);
       if (rc != ADADIM_OK) return rc;
-      if (tiles_after > 1) {
-        ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_block, 0));
-        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1,
-                          (tiles_after - 1 + rest_split - 1) / rest_split, status_dev, side);
+      const int tiles_after = static_cast<int>((in - i1 - kBlk) / kBlk);
+      if (tiles_after > 0) {
+        if (tiles_after > 1) ADADIM_CUDA_TRY(cudaEventRecord(ev_block, chain));
+        // the next block's columns were last written by the previous block's side-stream launch
+        if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
+        rest_pending = false;
+        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, 1, status_dev, chain);
         if (rc != ADADIM_OK) return rc;
-        ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
-        rest_pending = true;
+        if (tiles_after > 1) {
+          ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_block, 0));
+          rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1,
+                            (tiles_after - 1 + rest_split - 1) / rest_split, status_dev, side);
+          if (rc != ADADIM_OK) return rc;
+          ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
+          rest_pending = true;
+        }
       }
     }
+    for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k];
+    rc0 = fs.join();
+    if (rc0 != ADADIM_OK) return rc0;
   }
-  if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
-  ADADIM_CUDA_TRY(cudaEventRecord(ev_join, chain));
-  ADADIM_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
-  // destruction is deferred by the runtime until the work already enqueued has finished
-  cudaEventDestroy(ev_fork);
-  cudaEventDestroy(ev_block);
-  cudaEventDestroy(ev_rest);
-  cudaEventDestroy(ev_join);
-  cudaStreamDestroy(chain);
-  cudaStreamDestroy(side);
-  for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k];
   if (reorder) {
     const unsigned ub = static_cast<unsigned>((out * (in / 32) + 255) / 256);
     for (int d = 0; d < ndim; ++d) {

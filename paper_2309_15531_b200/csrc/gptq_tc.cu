@@ -10,7 +10,9 @@
 // bits, a sum of 128 of them has at most 23 bits, and the accumulation is exact: nothing is
 // left to truncate.  The leading products go to one TMEM accumulator, the five smaller
 // product classes (2^-8 and 2^-16 of the result) to a second one, and the two are added in
-// fp32 in the epilogue.
+// fp32 in the epilogue.  The working weights themselves are binary64 (gptq.cu says why): the
+// epilogue widens the negated product and hands it to the memory system as an element-wise
+// binary64 add, so the SM never reads W.
 //
 // One CTA owns a 128-row block of the stacked working weights and a range of 128-column
 // tiles.  Its Err pieces (K = 128) stay in shared memory; U pieces stream through a ring of
@@ -30,11 +32,11 @@ constexpr int kTileN = 128;
 constexpr uint32_t kBPiece = kTileN * 32 * 2;       // one U piece, 32 k-rows x 128 columns: 8 KB
 constexpr uint32_t kBStage = 3 * kBPiece;           // 24 KB
 constexpr int kBStages = 4;
-constexpr uint32_t kOutChunk = 32 * 32 * 4;          // one epilogue warp's staging tile: 32 rows x 32 fp32 columns
+constexpr uint32_t kOutChunk = 32 * 16 * 8;          // one epilogue warp's staging tile: 32 rows x 16 fp64 columns
 constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 8 * kOutChunk + 1024 + 256;
 
 struct TrailParams {
-  float* Wc;            // [rows_total][in] stacked working weights
+  double* Wc;           // stacked working weights, rows_total x in, in the tiled layout of wc_index()
   int64_t in;
   int64_t c0;           // first column to update
   int i1;               // first row of U's block
@@ -47,13 +49,12 @@ __global__ void __launch_bounds__(kThreads, 1)
 trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ CUtensorMap tmE1,
              const __grid_constant__ CUtensorMap tmE2, const __grid_constant__ CUtensorMap tmU0,
              const __grid_constant__ CUtensorMap tmU1, const __grid_constant__ CUtensorMap tmU2,
-             const __grid_constant__ CUtensorMap tmW,
              const TrailParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_smem = smem;
   uint8_t* b_smem = smem + kABytes;
-  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][32 rows][128 B], 128-byte swizzle
+  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][32 rows][128 B]
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 8 * kOutChunk);
   uint64_t* a_full = bars;
   uint64_t* b_full = bars + 1;                      // [kBStages]
@@ -173,36 +174,42 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
     }
   } else {
     // Two warps per TMEM lane quadrant, each taking one 64-column half of every tile.  W is never
-    // read here: the negated product goes to a staging tile in shared memory and from there into
-    // W as an element-wise add done by the memory system (W + (-p) is the same binary32 operation
-    // as W - p), 32 rows x 32 columns at a time, so the epilogue only issues writes.
+    // read here: 32 rows x 16 columns of the negated product, widened to binary64, are laid out in
+    // a staging tile exactly as a tile of the working weights is laid out in memory (wc_index) and
+    // handed to the memory system as one 4 KB element-wise add into that tile (W + (-p) is the same
+    // operation as W - p), so the epilogue only issues writes.
     const int q = warp & 3, half = (warp - 2) >> 2;
     uint32_t acc_phase[2] = {0, 0};
     uint8_t* stage_tile = out_smem + (warp - 2) * kOutChunk;
     uint8_t* my_row = stage_tile + lane * 128;        // this lane's row of the staging tile
+    // first tile of this warp's rows and of the launch's first column
+    double* wtile = p.Wc + (static_cast<int64_t>((mrow + q * 32) / kWcTileRows) * (p.in / kWcTileCols) +
+                            (p.c0 + half * 64) / kWcTileCols) * kWcTileElems;
     for (int t = t0; t < t1; ++t) {
       const int buf = (t - t0) & 1;
       if (!ptx::mbar_wait(&acc_full[buf], acc_phase[buf], dead, p.status_dev)) break;
       ptx::tc_fence_after_sync();
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        float v[32], v2[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + half * 64 + c * 32;
-        ptx::tmem_ld32(taddr, v);
-        ptx::tmem_ld32(taddr + kTileN, v2);
+      for (int c = 0; c < 4; ++c) {
+        float v[16], v2[16];
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * 256 + half * 64 + c * 16;
+        ptx::tmem_ld16_nowait(taddr, v);
+        ptx::tmem_ld16_nowait(taddr + kTileN, v2);
+        ptx::tmem_ld_wait();
         if (lane == 0) ptx::bulk_wait_read();         // the previous add has finished reading the staging tile
         __syncwarp();
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {                  // 16-byte chunk k of the row sits at chunk k ^ (row % 8)
-          float4 x;
-          x.x = -(v[4 * k] + v2[4 * k]);         x.y = -(v[4 * k + 1] + v2[4 * k + 1]);
-          x.z = -(v[4 * k + 2] + v2[4 * k + 2]); x.w = -(v[4 * k + 3] + v2[4 * k + 3]);
-          *reinterpret_cast<float4*>(my_row + ((k ^ (lane & 7)) << 4)) = x;
+        for (int k = 0; k < 8; ++k) {                  // column pair k of the row sits at pair position k ^ (row % 8)
+          double2 x;
+          x.x = -(static_cast<double>(v[2 * k]) + static_cast<double>(v2[2 * k]));
+          x.y = -(static_cast<double>(v[2 * k + 1]) + static_cast<double>(v2[2 * k + 1]));
+          *reinterpret_cast<double2*>(my_row + ((k ^ (lane & 7)) << 4)) = x;
         }
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) {
-          ptx::tma_reduce_add_2d(&tmW, static_cast<int>(p.c0) + t * kTileN + half * 64 + c * 32, mrow + q * 32, stage_tile);
+          ptx::bulk_reduce_add_f64(wtile + (static_cast<int64_t>(t) * (kTileN / kWcTileCols) + c) * kWcTileElems, stage_tile,
+                                   kOutChunk);
           ptx::bulk_commit();
         }
       }
@@ -249,16 +256,16 @@ __device__ __forceinline__ void slice3(float x, SliceGrid s, __nv_bfloat16& p0, 
 // U pieces: one grid per (128-row block b, column c).  Only columns right of the block are
 // ever read by the trailing update, so only those are written.
 __global__ void __launch_bounds__(128)
-slice_u_kernel(const float* __restrict__ U, int64_t in, __nv_bfloat16* __restrict__ p0, __nv_bfloat16* __restrict__ p1,
+slice_u_kernel(const double* __restrict__ U, int64_t in, __nv_bfloat16* __restrict__ p0, __nv_bfloat16* __restrict__ p1,
                __nv_bfloat16* __restrict__ p2) {
   const int b = blockIdx.y;
   if (static_cast<int>(blockIdx.x) <= b) return;
   const int64_t c = static_cast<int64_t>(blockIdx.x) * 128 + threadIdx.x;
-  const float* src = U + static_cast<int64_t>(b) * 128 * in + c;
+  const double* src = U + static_cast<int64_t>(b) * 128 * in + c;
   float v[128];
   float m = 0.0f;
 #pragma unroll
-  for (int i = 0; i < 128; ++i) { v[i] = src[static_cast<int64_t>(i) * in]; m = fmaxf(m, fabsf(v[i])); }
+  for (int i = 0; i < 128; ++i) { v[i] = static_cast<float>(src[static_cast<int64_t>(i) * in]); m = fmaxf(m, fabsf(v[i])); }
   const SliceGrid sg = slice_grid(m);
 #pragma unroll
   for (int i = 0; i < 128; ++i) {
@@ -274,19 +281,19 @@ slice_u_kernel(const float* __restrict__ U, int64_t in, __nv_bfloat16* __restric
 // Host-side state of one GPTQ call's trailing updates: the six tensor maps never change
 // between blocks, only the coordinates do.
 struct TrailPlan {
-  CUtensorMap e[3], u[3], w;
-  float* Wc;
+  CUtensorMap e[3], u[3];
+  double* Wc;
   int64_t rows_total, in;
   int sm_count;
 };
 
-int trail_split_u(const float* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st) {
+int trail_split_u(const double* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st) {
   const unsigned nb = static_cast<unsigned>(in / 128);
   if (nb > 1) slice_u_kernel<<<dim3(nb, nb - 1), 128, 0, st>>>(U, in, u0, u1, u2);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 
-int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
+int trail_plan(TrailPlan* plan, double* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
                const __nv_bfloat16* const u[3]) {
   plan->Wc = Wc;
   plan->rows_total = rows_total;
@@ -296,11 +303,6 @@ int trail_plan(TrailPlan* plan, float* Wc, int64_t rows_total, int64_t in, const
     if (rc != ADADIM_OK) return rc;
     rc = make_tmap_bf16(&plan->u[k], u[k], static_cast<uint64_t>(in), static_cast<uint64_t>(in),
                         static_cast<uint64_t>(in) * 2, 32);
-    if (rc != ADADIM_OK) return rc;
-  }
-  {
-    int rc = make_tmap_f32(&plan->w, Wc, static_cast<uint64_t>(in), static_cast<uint64_t>(rows_total),
-                           static_cast<uint64_t>(in) * 4, 32);
     if (rc != ADADIM_OK) return rc;
   }
   int dev = 0;
@@ -329,7 +331,7 @@ int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int tile
   int nsplit = (ntiles + tiles_per_cta - 1) / tiles_per_cta;
   if (nsplit < 1) nsplit = 1;
   trail_kernel<<<dim3(nsplit, mblocks), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],
-                                                                      plan.u[1], plan.u[2], plan.w, p);
+                                                                      plan.u[1], plan.u[2], p);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 

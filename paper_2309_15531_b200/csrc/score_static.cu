@@ -7,8 +7,9 @@
 // implicit device synchronisation is unacceptable.  For them this file reserves a fixed
 // scratch array in the library's own device image and runs the same kernels on it.
 //
-// The array exists once per GPU that loads the library, from load until the process exits,
-// whether or not this entry point is ever called.
+// The array exists once per GPU that uses the library and stays until the process exits.  With
+// the CUDA runtime's lazy module loading it becomes resident on a device when its address is
+// first looked up there, i.e. at the first call of this entry point on that device.
 #include <mutex>
 
 #include "common.cuh"
@@ -56,31 +57,17 @@ int adadim_score_select_static(const void* W, int wdtype, int64_t out, int64_t i
                                double* err, int* chosen, int* status_dev, void* cuda_stream) {
   using namespace adadim;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  // the same argument rules as adadim_score_select
-  if (bits != 3 && bits != 4) return ADADIM_ERR_PARAM;
-  if (group != 32 && group != 64 && group != 128) return ADADIM_ERR_PARAM;
-  if (out <= 0 || in <= 0 || ldw < in) return ADADIM_ERR_SHAPE;
-  if (W == nullptr || H == nullptr || err == nullptr || chosen == nullptr) return ADADIM_ERR_NULL;
-  if (wdtype != ADADIM_F16 && wdtype != ADADIM_F32) return ADADIM_ERR_DTYPE;
-  if (!aligned16(W) || (ldw * (wdtype == ADADIM_F16 ? 2 : 4)) % 16 != 0 || !aligned16(H)) return ADADIM_ERR_ALIGN;
-  if (in % 64 != 0 || out % 128 != 0) return ADADIM_ERR_SHAPE;
-  if (q_oc == nullptr && q_ic == nullptr) return ADADIM_ERR_NULL;
-  const adadim_qtensor* qs[2] = {q_oc, q_ic};
-  for (int d = 0; d < 2; ++d) {
-    if (qs[d] == nullptr) continue;
-    if (qs[d]->codes == nullptr || qs[d]->scales == nullptr || qs[d]->zeros == nullptr) return ADADIM_ERR_NULL;
-    if (!aligned16(qs[d]->codes) || !aligned16(qs[d]->scales) || !aligned16(qs[d]->zeros)) return ADADIM_ERR_ALIGN;
-    if ((d == 0 ? in : out) % group != 0) return ADADIM_ERR_SHAPE;
-  }
+  // the same argument rules as adadim_score_select, checked by the same function
+  int rc = check_score_args(W, wdtype, out, in, ldw, H, bits, group, q_oc, q_ic, err, chosen);
+  if (rc != ADADIM_OK) return rc;
   // the size limit: the layer's scoring workspace must fit the built-in array
   if (score_workspace_bytes(out, in) > ADADIM_STATIC_SCRATCH_BYTES) return ADADIM_ERR_WORKSPACE;
   void* scratch = nullptr;
-  int rc = scratch_address(&scratch);
+  rc = scratch_address(&scratch);
   if (rc != ADADIM_OK) return rc;
-  if (status_dev != nullptr && cudaMemsetAsync(status_dev, 0, sizeof(int), st) != cudaSuccess) return ADADIM_ERR_CUDA;
   // Nothing in the scratch has to start at zero: every region the kernels read (the weight
-  // differences, the two halves of H, the per-tile partial sums) is fully rewritten by this
-  // call before it is read, so whatever an earlier call left behind is never observed.
+  // differences and the per-tile partial sums) is fully rewritten by this call before it is
+  // read, so whatever an earlier call left behind is never observed.
   return score_launch(W, wdtype, out, in, ldw, H, bits, group, q_oc, q_ic, err, chosen, status_dev, scratch, st);
 }
 

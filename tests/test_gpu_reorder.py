@@ -130,34 +130,37 @@ def test_reordered_flow_matches_the_oracle_flow():
 
 
 def test_reordered_full_size_layer():
-    """4096 x 4096 (q_proj recipe, 16384 tokens, activation magnitudes spread so that the order is
-    far from natural).  Against the oracle on one 128-row slab: the columns quantized first (where
-    rounding order has not yet had its say) within the strict bound, the errors of the slab within
-    1e-3.  Over the whole layer: the loss identity 1/2 sum(e^2) = 1/2 trace(D Hd D^T), which a wrong
-    gather, update or un-permutation breaks, and the per-OC parameters bit-exact (static groups)."""
-    wl = I.workload_qproj(n_tokens=16384)
+    """4096 x 4096 (q_proj recipe at its full 128 x 2048 tokens, activation magnitudes spread so
+    that the order is far from natural; the Hessian is summed in binary64 on the device).  Against the oracle on one 128-row slab: every column at the stated bar
+    (<= 0.1 % of codes, <= 1 level), the errors of the slab within 1e-3.  Over the whole layer: the
+    loss identity 1/2 sum(e^2) = 1/2 trace(D Hd D^T), which a wrong gather, update or
+    un-permutation breaks, and the per-OC parameters bit-exact (static groups)."""
+    wl = I.workload_qproj()
     wspec, xspec = wl["layers"]["q_proj"]
     W = I.make_weight(wspec, "cuda")
-    X = I.make_calib(xspec, "cuda")
     g = torch.Generator(device="cuda").manual_seed(71)
-    X = (X.float() * (0.5 + 1.5 * torch.rand(4096, device="cuda", generator=g))).bfloat16()
+    spread = 0.5 + 1.5 * torch.rand(4096, device="cuda", generator=g)
+    X = I.make_calib(xspec, "cuda")
+    H64 = torch.zeros(4096, 4096, dtype=torch.float64, device="cuda")
+    for t0 in range(0, xspec.n_tokens, 16384):
+        Xc = (X[t0:t0 + 16384].float() * spread).bfloat16().double()
+        H64.addmm_(Xc.T, Xc, alpha=2.0)
+    del X
     Wn = to_np(W).astype(np.float32)
-    Hn = O.hessian(to_np(X)).astype(np.float32)
+    Hn = H64.float().cpu().numpy()
     q_oc, q_ic, loss, perm = _run(W, Hn, 3, 128)
     assert np.array_equal(perm, O.activation_order(Hn.astype(np.float64)))
     rows = slice(1280, 1408)
-    first = perm[:1024]
     for k, (name, q) in enumerate((("oc", q_oc), ("ic", q_ic))):
         codes, s, z = q_to_np(q)
         # the oracle on the slab needs the whole-matrix static parameters only for its own rows
         ref = O.quantize_gptq_reordered(Wn[rows], Hn, 3, 128, name, 0.01, static_groups=(name == "oc"))
-        frac, lvl = code_mismatch(codes[rows][:, first], ref["codes"][:, first])
-        frac_all, _ = code_mismatch(codes[rows], ref["codes"])
+        frac, lvl = code_mismatch(codes[rows], ref["codes"])
         Q = O.dequantize(codes, s, z, 128, name)
         e_gpu = O.recon_error_trace(Wn[rows], Q[rows], Hn.astype(np.float64))
         e_ref = O.recon_error_trace(Wn[rows], ref["Q"], Hn.astype(np.float64))
-        print(f"reordered full-size {name}: first 1024 columns differ {100 * frac:.4f}% (max {lvl}), "
-              f"all columns {100 * frac_all:.3f}%, E gpu {e_gpu:.6e} oracle {e_ref:.6e}")
+        print(f"reordered full-size {name}: codes differ {100 * frac:.4f}% (max {lvl}), "
+              f"E gpu {e_gpu:.6e} oracle {e_ref:.6e}")
         assert frac <= 1e-3 and lvl <= 1
         assert e_gpu == pytest.approx(e_ref, rel=1e-3)
         if name == "oc":

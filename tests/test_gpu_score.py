@@ -88,6 +88,29 @@ def test_tie_gives_oc_and_nan_is_reported():
     assert int(st.item()) == 8 and int(chosen.item()) == B.DIM_OC
 
 
+def test_status_word_is_sticky_across_calls():
+    """A device-side condition reported by one call survives later successful calls that are
+    given the same status word: the caller may check once after a whole sequence."""
+    W = torch.zeros(128, 128, dtype=torch.float16, device="cuda")
+    W[:, 3] = 0.013
+    Hbad = torch.eye(128, device="cuda")
+    Hbad[3, 3] = float("nan")
+    Hgood = torch.eye(128, device="cuda")
+    q_oc, q_ic = B.quantize_rtn(W, 3, 128)
+    st = status_tensor()
+    B.score_select(W, Hbad, 3, 128, q_oc, q_ic, status=st)            # reports ADADIM_ERR_NUMERIC
+    err, _ = B.score_select(W, Hgood, 3, 128, q_oc, q_ic, status=st)  # a clean call afterwards
+    X = I.make_calib(I.CalibSpec(256, 128, "bf16", "normal", 0, seed=59), "cuda")
+    B.hessian_accumulate(X, torch.zeros(128, 128, device="cuda"), st)
+    B.quantize_gptq(W, Hgood, 3, 128, B.DIM_BOTH, status=st)
+    torch.cuda.synchronize()
+    assert np.isfinite(err.cpu().numpy()).all()
+    assert int(st.item()) == 8
+    st.zero_()                                                        # the caller clears it
+    B.score_select(W, Hgood, 3, 128, q_oc, q_ic, status=st)
+    assert int(st.item()) == 0
+
+
 def test_workspace_too_small_is_refused():
     W = torch.zeros(128, 128, dtype=torch.float16, device="cuda")
     H = torch.eye(128, device="cuda")
