@@ -3,10 +3,13 @@
 
 One step = one pass of the whole path over one layer: calibration Hessian over all tokens,
 RTN in both grouping dimensions, score + select, damped Cholesky-inverse factor, GPTQ in both
-dimensions, score + select.  Workload: the LLaMA-7B q_proj-shaped layer (W 4096 x 4096 fp16,
-X 262144 x 4096 bf16), 3-bit, group 128, seeded synthetic tensors.
+dimensions, score + select.  Default workload (the one the metric is quoted on): the LLaMA-7B
+q_proj-shaped layer (W 4096 x 4096 fp16, X 262144 x 4096 bf16), 3-bit, group 128, seeded
+synthetic tensors.  `--workload down_proj | block | mlp70b` times the other benchmark
+configurations (one step = every layer and variant of that configuration once); they report the
+same keys per layer and for the whole set, without the host-buffer leg.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 Prints one JSON line.  With N > 1 (under torchrun) every rank quantizes its own replica of the
 layer; there is no data-path collective.  `--impl reference` times the CPU oracle on a bounded
@@ -28,6 +31,7 @@ if ROOT not in sys.path:
 
 METRIC = "AdaDim layer quant weights/s (RTN & GPTQ, 3b g128); % of HBM/tensor roofline"
 BITS, GROUP = 3, 128
+DTYPE = "bf16 (Hessian and scorer: bf16 tensor cores, fp32 accumulation); f32 (quantizer); f64 (factor, GPTQ)"
 WORKLOAD = ("llama7b_q_proj W[4096,4096] fp16, X[262144,4096] bf16, 3-bit g128, "
             "Hessian + RTN both dims + score + factor + GPTQ both dims + score")
 
@@ -39,6 +43,66 @@ def _peaks():
         return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
                 "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def stage_rooflines(stage_ms, out, inp, ntok, bits, group, peaks, mhz, clocks):
+    """What bounds each stage of one layer's pass, from the stage's CUDA-event time.
+    Tensor-core stages are given against both measured bf16 figures: the burst one applies when the
+    SM clock stayed at its maximum with no power cap during the timed region, the sustained one
+    when sw_power_cap was active; `frac` follows whichever applies."""
+    tile = 256
+    weights = out * inp
+    capped = bool(clocks and "sw_power_cap" in (clocks.get("reasons") or []))
+    r = {}
+
+    def tensor(name, flops):
+        ach = flops / (stage_ms[name] * 1e-3) / 1e12
+        r[name] = {"bound": "tensor", "achieved": ach, "unit": "TFLOP/s",
+                   "peak": peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"],
+                   "peak_source": peaks["source"] + (" (sustained bf16: power cap active)" if capped
+                                                      else " (burst bf16: full clock, no cap)"),
+                   "frac_of_burst": ach / peaks["bf16_tflops"], "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
+        r[name]["frac"] = r[name]["frac_of_sustained"] if capped else r[name]["frac_of_burst"]
+
+    if "hessian" in stage_ms:
+        tensor("hessian", ntok * inp * (inp + tile))          # lower-triangle tiles of the symmetric product
+    for name in ("score_rtn", "score_gptq"):
+        if name in stage_ms:
+            tensor(name, 2 * out * inp * (inp + tile))        # D^T D on lower-triangle tiles, both dims
+    if "rtn" in stage_ms:
+        ach = weights * (2 + 2 * (bits / 8 + 4 / group)) / (stage_ms["rtn"] * 1e-3) / 1e9
+        r["rtn"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "peak_source": peaks["source"], "frac": ach / peaks["hbm_gbs"]}
+    if "factor" in stage_ms:
+        ach = 2 * inp ** 3 / 3 / (stage_ms["factor"] * 1e-3) / 1e12       # Cholesky + triangular inverse
+        pk = 148 * 64 * 2 * mhz * 1e6 / 1e12
+        r["factor"] = {"bound": "alu", "achieved": ach, "peak": pk, "unit": "TFLOP/s", "frac": ach / pk,
+                       "note": "fp64 FMA: 148 SMs x 64 FMA/clk x 2 at the sampled SM clock"}
+    if "gptq" in stage_ms:
+        blocks = inp // 128
+        r["gptq"] = {"bound": "latency", "ms": stage_ms["gptq"], "column_blocks": blocks,
+                     "us_per_column_block": stage_ms["gptq"] * 1e3 / blocks,
+                     "cycles_per_column": stage_ms["gptq"] * 1e-3 * mhz * 1e6 / inp,
+                     "note": "a chain of `column_blocks` block kernels, each 128 dependent column steps; the "
+                             "tensor-core trailing updates run beside it on a second stream"}
+    return r
+
+
+def measured_traffic(name):
+    """DRAM bytes of one launch of the dominant kernel from the ncu capture kept beside its
+    profile summary; null once the kernel's sources differ from the ones the capture was taken with."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", name + ".traffic.json")
+    if not os.path.exists(path):
+        return {"traffic": None, "traffic_note": "no capture on file"}
+    d = json.load(open(path))
+    h = hashlib.sha256()
+    for f in d["sources"]:
+        h.update(open(os.path.join(ROOT, f), "rb").read())
+    if h.hexdigest() != d["sources_sha256"]:
+        return {"traffic": None, "traffic_note": "kernel sources changed since the capture"}
+    return {"traffic": d["dram_bytes_read"] + d["dram_bytes_write"], "traffic_unit": d["unit"],
+            "traffic_algorithmic": d["algorithmic_bytes"], "traffic_note": d["note"]}
 
 
 # --------------------------------------------------------------------------- clocks sampler
@@ -88,8 +152,8 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- launch count
-def launches_per_step(out: int, inp: int) -> int:
-    """Kernels of this library launched by one step (mirrors the host-side launch logic)."""
+def launches_hessian_factor(inp: int) -> int:
+    """Kernels launched by one Hessian accumulation plus one factor (mirrors the host-side launch logic)."""
     nb = inp // 64
     factor = 2                                           # damping, build
     for g0 in range(0, nb, 4):
@@ -104,12 +168,21 @@ def launches_per_step(out: int, inp: int) -> int:
         factor += 2
         s *= 2
     factor += 1                                          # emit
+    hessian = 2 if inp > 256 else 1
+    return hessian + factor
+
+
+def launches_layer(inp: int, score_gptq: bool = True) -> int:
+    """Kernels launched for one layer: RTN, scoring, GPTQ (with a precomputed factor), scoring."""
     blocks = inp // 128
     gptq = 1 + 1 + blocks + (blocks - 1) + max(blocks - 2, 0) + 1   # init, U slicing, block kernels, next-block and rest trailing kernels, loss
-    hessian = 2 if inp > 256 else 1
     rtn = 1
     score = 1 + 1 + 1                                  # difference kernel, Gram product, finalize
-    return hessian + rtn + score + factor + gptq + score
+    return rtn + score + gptq + (score if score_gptq else 0)
+
+
+def launches_per_step(out: int, inp: int) -> int:
+    return launches_hessian_factor(inp) + launches_layer(inp)
 
 
 # --------------------------------------------------------------------------- rank aggregation
@@ -168,8 +241,8 @@ def run_ours(args):
         def mark(i):
             if ev is not None:
                 ev[i].record()
-        H.zero_()
         mark(0)
+        H.zero_()
         B.hessian_accumulate(Xd, H, st)
         mark(1)
         B.quantize_rtn(Wd, BITS, GROUP, B.DIM_BOTH, r_oc, r_ic)
@@ -312,48 +385,23 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel ---------------------------------------------------------
+    # ---- rooflines -------------------------------------------------------------------------------
     peaks = _peaks()
-    tile = 256
-    hess_flops = ntok * inp * (inp + tile)              # lower-triangle tiles of the symmetric product
-    rtn_bytes = weights * (2 + 2 * (BITS / 8 + 4 / GROUP))
-    score_flops = 2 * out * inp * (inp + tile)           # D^T D on lower-triangle tiles, both dims
-    factor_flops = 2 * inp ** 3 / 3                     # Cholesky + triangular inverse
-    gptq_flops = 2 * (out * inp * inp)                  # trailing + in-block updates, both dims
-    roof_all = {
-        "hessian": {"bound": "tensor", "achieved": hess_flops / (stage_ms["hessian"] * 1e-3) / 1e12,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"},
-        "rtn": {"bound": "hbm", "achieved": rtn_bytes / (stage_ms["rtn"] * 1e-3) / 1e9,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s"},
-        "score_rtn": {"bound": "tensor", "achieved": score_flops / (stage_ms["score_rtn"] * 1e-3) / 1e12,
-                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"},
-    }
     mhz = (clocks or {}).get("sm_mhz") or 1965.0
-    roof_all["factor"] = {"bound": "alu", "achieved": factor_flops / (stage_ms["factor"] * 1e-3) / 1e12,
-                          "peak": 148 * 64 * 2 * mhz * 1e6 / 1e12, "unit": "TFLOP/s",
-                          "note": "fp64 FMA: 148 SMs x 64 FMA/clk x 2 at the sampled SM clock"}
-    roof_all["gptq"] = {"bound": "alu", "achieved": gptq_flops / (stage_ms["gptq"] * 1e-3) / 1e12,
-                        "peak": 148 * 128 * 2 * mhz * 1e6 / 1e12, "unit": "TFLOP/s",
-                        "note": "sequential depth = in; fp32 FMA peak at the sampled SM clock for scale only"}
-    for v in roof_all.values():
-        v["frac"] = v["achieved"] / v["peak"]
+    roof_all = stage_rooflines(stage_ms, out, inp, ntok, BITS, GROUP, peaks, mhz, clocks)
     # The dominant kernel is the Hessian's tensor-core kernel (the factor and GPTQ stages are longer
-    # but are sequences of short launches).  Its time is the hessian stage's CUDA-event time (tc kernel
-    # + the 24 us mirror copy); traffic is dram read + write of that launch from ncu
-    # (profiles/tensor_core_kernels_llama7b_q_proj.md), taken with this kernel as it stands.
+    # but are sequences of short launches).  Its time is the hessian stage's CUDA-event time (zeroing
+    # H + the tensor-core kernel + the 24 us mirror copy).
     roofline = dict(roof_all["hessian"])
     roofline["kernel"] = "tc_kernel<Hessian>"
-    roofline["peak_source"] = peaks["source"] + " (sustained bf16)"
-    roofline["traffic"] = 4.372e9 + 1.091e9
-    roofline["traffic_unit"] = ("bytes per launch (algorithmic: 2.147e9 of X + 1.08e9 written and as much read by the "
-                                "memory system for the 32 element-wise adds into H)")
+    roofline.update(measured_traffic("tc_kernel_hessian_llama7b_q_proj"))
 
     cpu = None if args.no_cpu_baseline else cpu_baseline()
 
     line = {
         "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": WORKLOAD,
                    "l2": "flushed between steps by writing a 256 MiB buffer; X (2.1 GB) exceeds L2",
                    "replicas": world},
@@ -367,6 +415,178 @@ def run_ours(args):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- the other configurations
+def config_jobs(name):
+    """(workload dict, list of (layer name, [(bits, group, mode)])) for a benchmark configuration.
+    mode "both": RTN in both dimensions + score, GPTQ in both dimensions + score + select.
+    mode "ada":  the paper's flow: RTN in both dimensions + score + select, GPTQ in the chosen one."""
+    from paper_2309_15531_b200 import inputs as I
+    if name == "down_proj":
+        wl = I.workload_downproj()
+        return wl, [("down_proj", [(b, g, "both") for b, g in wl["variants"]])]
+    if name == "block":
+        wl = I.workload_block()
+        return wl, [(n, [(3, 128, "ada")]) for n in wl["layers"]]
+    if name == "mlp70b":
+        wl = I.workload_mlp70b()
+        return wl, [(n, [(4, 128, "both")]) for n in wl["layers"]]
+    raise ValueError(name)
+
+
+def run_config(args):
+    """One step = every Hessian, factor, layer and variant of the configuration once.  Layers that
+    share an input width share one activation tensor, one Hessian and one factor."""
+    import torch
+    from paper_2309_15531_b200 import binding as B
+    from paper_2309_15531_b200 import inputs as I
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return                                            # one replica is enough for these lines
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl, jobs = config_jobs(args.workload)
+    xspecs = {}
+    for lname, _ in jobs:
+        xs = wl["layers"][lname][1]
+        xspecs.setdefault(xs, []).append(lname)
+    Ws = {n: I.make_weight(wl["layers"][n][0], dev) for n, _ in jobs}
+    Xs = {xs: I.make_calib(xs, dev) for xs in xspecs}
+    Hs = {xs: torch.zeros(xs.inp, xs.inp, device=dev) for xs in xspecs}
+    Us = {xs: torch.empty(xs.inp, xs.inp, dtype=torch.float64, device=dev) for xs in xspecs}
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    max_g = max(B.workspace_bytes(B.WS_GPTQ, w.out, w.inp) for w, _ in wl["layers"].values())
+    max_s = max(B.workspace_bytes(B.WS_SCORE, w.out, w.inp) for w, _ in wl["layers"].values())
+    max_f = max(B.workspace_bytes(B.WS_FACTOR, 0, xs.inp) for xs in xspecs)
+    ws_g = torch.empty(max_g, dtype=torch.uint8, device=dev)
+    ws_s = torch.empty(max_s, dtype=torch.uint8, device=dev)
+    ws_f = torch.empty(max_f, dtype=torch.uint8, device=dev)
+    q = {}
+    for lname, variants in jobs:
+        w = wl["layers"][lname][0]
+        for bits, group, _ in variants:
+            q[(lname, bits, group)] = [B.QTensor(w.out, w.inp, bits, group, d, dev)
+                                       for d in (B.DIM_OC, B.DIM_IC, B.DIM_OC, B.DIM_IC)]
+    err_r = torch.zeros(2, dtype=torch.float64, device=dev)
+    err_g = torch.zeros(2, dtype=torch.float64, device=dev)
+    ch_r = torch.zeros(1, dtype=torch.int32, device=dev)
+    ch_g = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    chosen = {}
+
+    def one_step(rec):
+        def timed(key, fn):
+            if rec is None:
+                fn()
+                return
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            rec.append((key, e0, e1))
+        for xs in xspecs:
+            def hess(xs=xs):
+                Hs[xs].zero_()
+                B.hessian_accumulate(Xs[xs], Hs[xs], st)
+            timed(("hessian", xs.inp), hess)
+            timed(("factor", xs.inp), lambda xs=xs: lib_factor(B, Hs[xs], Us[xs], st, ws_f))
+        for lname, variants in jobs:
+            W = Ws[lname]
+            xs = wl["layers"][lname][1]
+            H, U = Hs[xs], Us[xs]
+            for bits, group, mode in variants:
+                r_oc, r_ic, g_oc, g_ic = q[(lname, bits, group)]
+                timed(("rtn", lname, bits, group), lambda: B.quantize_rtn(W, bits, group, B.DIM_BOTH, r_oc, r_ic))
+                timed(("score_rtn", lname, bits, group),
+                      lambda: B.score_select(W, H, bits, group, r_oc, r_ic, err_r, ch_r, st, ws_s))
+                if mode == "both":
+                    timed(("gptq", lname, bits, group),
+                          lambda: B.quantize_gptq(W, H, bits, group, B.DIM_BOTH, 0.01, U, g_oc, g_ic, None, st, ws_g))
+                    timed(("score_gptq", lname, bits, group),
+                          lambda: B.score_select(W, H, bits, group, g_oc, g_ic, err_g, ch_g, st, ws_s))
+                    chosen[(lname, bits, group)] = ch_g.clone()
+                else:
+                    dim = int(ch_r.item())               # the one read-back per layer: it decides what runs next
+                    chosen[(lname, bits, group)] = dim
+                    timed(("gptq", lname, bits, group),
+                          lambda: B.quantize_gptq(W, H, bits, group, dim, 0.01, U,
+                                                  g_oc if dim == B.DIM_OC else None,
+                                                  g_ic if dim == B.DIM_IC else None, None, st, ws_g))
+
+    for _ in range(max(args.warmup, 1)):
+        one_step(None)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0, f"device status {int(st.item())}"
+    sampler = ClockSampler(0)
+    sampler.start()
+    recs, whole = [], []
+    t0 = time.time()
+    for k in range(args.steps):
+        flush.fill_(k & 0xFF)
+        rec = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); one_step(rec); e1.record()
+        recs.append(rec); whole.append((e0, e1))
+    torch.cuda.synchronize()
+    clocks = sampler.stop(t0, time.time())
+    assert int(st.item()) == 0, f"device status {int(st.item())}"
+    ms_per_step = sum(a.elapsed_time(b) for a, b in whole) / args.steps
+    ms = {}
+    for rec in recs:
+        for key, a, b in rec:
+            ms[key] = ms.get(key, 0.0) + a.elapsed_time(b) / args.steps
+
+    peaks = _peaks()
+    mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    ntok = next(iter(xspecs)).n_tokens
+    weights_total = sum(w.out * w.inp for w, _ in wl["layers"].values())
+    hess_ms = sum(v for k, v in ms.items() if k[0] == "hessian")
+    layers = {}
+    for lname, variants in jobs:
+        w = wl["layers"][lname][0]
+        for bits, group, mode in variants:
+            stage = {k[0]: v for k, v in ms.items() if k[1:] == (lname, bits, group)}
+            roof = stage_rooflines(stage, w.out, w.inp, ntok, bits, group, peaks, mhz, clocks)
+            t_layer = sum(stage.values())
+            c = chosen[(lname, bits, group)]
+            layers[f"{lname} {bits}b g{group}"] = {
+                "shape": [w.out, w.inp], "flow": mode, "stages_ms": stage, "ms": t_layer,
+                "weights_per_s": w.out * w.inp / (t_layer * 1e-3),
+                "chosen": B.DIM_NAMES[int(c.item()) if hasattr(c, "item") else c], "rooflines": roof}
+    shared = {}
+    for xs in xspecs:
+        stage = {"hessian": ms[("hessian", xs.inp)], "factor": ms[("factor", xs.inp)]}
+        shared[f"in={xs.inp} ({', '.join(xspecs[xs])})"] = {
+            "stages_ms": stage, "rooflines": stage_rooflines(stage, 0, xs.inp, xs.n_tokens, 0, 1, peaks, mhz, clocks)}
+    n_var = sum(len(v) for _, v in jobs)
+    # the dominant kernel of these configurations too is the Hessian's tensor-core kernel
+    big = max(xspecs, key=lambda xs: xs.inp)
+    roofline = dict(shared[f"in={big.inp} ({', '.join(xspecs[big])})"]["rooflines"]["hessian"])
+    roofline["kernel"] = f"tc_kernel<Hessian>, in={big.inp}"
+    roofline["traffic"] = None
+    line = {
+        "metric": METRIC, "value": weights_total / (ms_per_step * 1e-3), "unit": "weights/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+        "config": {"workload": f"{wl['name']}: {len(jobs)} layer(s), {n_var} layer-variant(s), {ntok} calibration tokens; "
+                               "one Hessian and one factor per distinct input width",
+                   "l2": "flushed between steps by writing a 256 MiB buffer; every X exceeds L2", "replicas": 1},
+        "ms_per_step_without_hessians": ms_per_step - hess_ms,
+        "weights_per_s_without_hessians": weights_total / ((ms_per_step - hess_ms) * 1e-3),
+        "layers": layers, "shared": shared, "roofline": roofline, "cpu_baseline": None,
+        "e2e": None, "e2e_note": "the host-buffer leg is measured on the default workload only",
+        "clocks": clocks,
+        "gpu_launches": args.steps * (sum(launches_hessian_factor(xs.inp) for xs in xspecs) +
+                                      sum(launches_layer(wl["layers"][n][0].inp, m == "both")
+                                          for n, v in jobs for _, _, m in v)),
+    }
+    print(json.dumps(line))
+
+
+def lib_factor(B, H, U, st, ws_f):
+    """adadim_cholesky_inverse_factor into a preallocated U."""
+    rc = B.lib().adadim_cholesky_inverse_factor(H.data_ptr(), H.shape[0], 0.01, U.data_ptr(), st.data_ptr(),
+                                                ws_f.data_ptr(), ws_f.numel(), B._stream())
+    B._check(rc, "adadim_cholesky_inverse_factor")
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
@@ -438,11 +658,14 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="q_proj", choices=["q_proj", "down_proj", "block", "mlp70b"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "q_proj":
+        run_config(args)
     else:
         run_ours(args)
 

@@ -8,9 +8,10 @@
 // and per U column of the block (x = p0 + p1 + p2, piece k a multiple of grid * 2^-8k).  Every
 // bf16 product of two leading pieces is then an integer multiple of one unit with at most 16
 // bits, a sum of 128 of them has at most 23 bits, and the accumulation is exact: nothing is
-// left to truncate.  The leading products go to one TMEM accumulator, the five smaller
-// product classes (2^-8 and 2^-16 of the result) to a second one, and the two are added in
-// fp32 in the epilogue.  The working weights themselves are binary64 (gptq.cu says why): the
+// left to truncate.  The leading products go to one TMEM accumulator, the eight smaller
+// products (2^-8 ... 2^-32 of the result) to a second one, and the two are added in binary64 in
+// the epilogue.  All nine products are formed: leaving out the three smallest (2^-24 of the
+// largest term) was measured to flip a rounding decision now and then on long layers.  The working weights themselves are binary64 (gptq.cu says why): the
 // epilogue widens the negated product and hands it to the memory system as an element-wise
 // binary64 add, so the SM never reads W.
 //
@@ -148,10 +149,10 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
 #pragma unroll
           for (int k16 = 0; k16 < 2; ++k16) {
 #pragma unroll
-            for (int pr = 0; pr < 6; ++pr) {
-              // (Err piece, U piece) with piece indices summing to at most 2
-              const int pa = pr == 0 ? 0 : pr == 1 ? 0 : pr == 2 ? 1 : pr == 3 ? 0 : pr == 4 ? 1 : 2;
-              const int pb = pr == 0 ? 0 : pr == 1 ? 1 : pr == 2 ? 0 : pr == 3 ? 2 : pr == 4 ? 1 : 0;
+            for (int pr = 0; pr < 9; ++pr) {
+              // all nine (Err piece, U piece) products, by falling magnitude: piece index sums 0, 1, 1, 2, 2, 2, 3, 3, 4
+              const int pa = pr == 0 ? 0 : pr == 1 ? 0 : pr == 2 ? 1 : pr == 3 ? 0 : pr == 4 ? 1 : pr == 5 ? 2 : pr == 6 ? 1 : 2;
+              const int pb = pr == 0 ? 0 : pr == 1 ? 1 : pr == 2 ? 0 : pr == 3 ? 2 : pr == 4 ? 1 : pr == 5 ? 0 : pr == 6 ? 2 : pr == 7 ? 1 : 2;
               // leading product -> exact accumulator; the rest -> the second one
               const uint32_t acc = tmem_base + buf * 256 + (pr == 0 ? 0 : kTileN);
               const bool first = (kc | k16) == 0 && pr <= 1;
