@@ -558,6 +558,33 @@ def run_config(args):
         shared[f"in={xs.inp} ({', '.join(xspecs[xs])})"] = {
             "stages_ms": stage, "rooflines": stage_rooflines(stage, 0, xs.inp, xs.n_tokens, 0, 1, peaks, mhz, clocks)}
     n_var = sum(len(v) for _, v in jobs)
+    block_flow = None
+    if args.workload == "block":
+        # the same block through flows.block_gptq_ada: layers that share an input run GPTQ stacked in one
+        # batched call, the dimension is read on the device, the factor runs beside RTN and scoring
+        from paper_2309_15531_b200 import flows
+        flow_layers = [(n, Ws[n], Xs[wl["layers"][n][1]]) for n, _ in jobs]
+        for _ in range(2):
+            res = flows.block_gptq_ada(flow_layers, 3, 128, status=st)
+        torch.cuda.synchronize()
+        t_flow = []
+        for k in range(args.steps):
+            flush.fill_(k & 0xFF)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            res = flows.block_gptq_ada(flow_layers, 3, 128, status=st)
+            e1.record()
+            torch.cuda.synchronize()
+            t_flow.append(e0.elapsed_time(e1))
+        assert int(st.item()) == 0, f"device status {int(st.item())}"
+        flow_ms = sum(t_flow) / len(t_flow)
+        same = all(int(res[n][0].item()) == (chosen[(n, 3, 128)]) for n, _ in jobs)
+        block_flow = {"ms_per_block": flow_ms, "ms_per_block_without_hessians": flow_ms - hess_ms,
+                      "weights_per_s": weights_total / (flow_ms * 1e-3),
+                      "weights_per_s_without_hessians": weights_total / ((flow_ms - hess_ms) * 1e-3),
+                      "same_choices_as_layer_by_layer": bool(same),
+                      "how": "flows.block_gptq_ada: q,k,v,o stacked in one batched GPTQ call (128 slabs), gate and up "
+                             "in one each... per max_stacked_rows; no host read-back between RTN selection and GPTQ"}
     # the dominant kernel of these configurations too is the Hessian's tensor-core kernel
     big = max(xspecs, key=lambda xs: xs.inp)
     roofline = dict(shared[f"in={big.inp} ({', '.join(xspecs[big])})"]["rooflines"]["hessian"])
@@ -572,7 +599,7 @@ def run_config(args):
                    "l2": "flushed between steps by writing a 256 MiB buffer; every X exceeds L2", "replicas": 1},
         "ms_per_step_without_hessians": ms_per_step - hess_ms,
         "weights_per_s_without_hessians": weights_total / ((ms_per_step - hess_ms) * 1e-3),
-        "layers": layers, "shared": shared, "roofline": roofline, "cpu_baseline": None,
+        "layers": layers, "shared": shared, "block_flow": block_flow, "roofline": roofline, "cpu_baseline": None,
         "e2e": None, "e2e_note": "the host-buffer leg is measured on the default workload only",
         "clocks": clocks,
         "gpu_launches": args.steps * (sum(launches_hessian_factor(xs.inp) for xs in xspecs) +

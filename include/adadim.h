@@ -60,9 +60,13 @@ typedef enum {
 } adadim_status;
 
 typedef enum { ADADIM_F32 = 0, ADADIM_F16 = 1, ADADIM_BF16 = 2 } adadim_dtype;
-typedef enum { ADADIM_DIM_OC = 0, ADADIM_DIM_IC = 1, ADADIM_DIM_BOTH = 2 } adadim_dim;
+/* ADADIM_DIM_CHOSEN (batched GPTQ only): the dimension is read from a device word at run time. */
+typedef enum { ADADIM_DIM_OC = 0, ADADIM_DIM_IC = 1, ADADIM_DIM_BOTH = 2, ADADIM_DIM_CHOSEN = 3 } adadim_dim;
+/* ADADIM_WS_GPTQ: one layer [out][in] in up to both dimensions.  ADADIM_WS_GPTQ_ROWS: `out` is the
+ * total number of working rows of a batched call (sum over its layers of out, twice for a layer
+ * quantized in both dimensions). */
 typedef enum { ADADIM_WS_HESSIAN = 0, ADADIM_WS_GPTQ = 1, ADADIM_WS_SCORE = 2,
-               ADADIM_WS_FACTOR = 3 } adadim_ws_kind;
+               ADADIM_WS_FACTOR = 3, ADADIM_WS_GPTQ_ROWS = 4 } adadim_ws_kind;
 
 /*
  * One quantized tensor (device pointers, caller-owned).
@@ -148,7 +152,8 @@ ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, double
  *   U          optional precomputed adadim_cholesky_inverse_factor of the same H, or NULL.
  *   blocksize  128.  group must divide 128 (32, 64, 128; 256 is refused with ADADIM_ERR_PARAM).
  *              in % 128 == 0, out % 128 == 0.
- *   gptq_loss  optional device double[2] (OC, IC): 1/2 * sum of e^2.
+ *   gptq_loss  optional device double[2] (OC, IC): 1/2 * sum of e^2 (only the element of a
+ *              dimension that was run is written).
  *   workspace  adadim_workspace_bytes(ADADIM_WS_GPTQ, out, in, bits, group), 256-byte aligned.
  */
 ADADIM_API int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
@@ -156,6 +161,44 @@ ADADIM_API int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int6
                          double percdamp, int blocksize,
                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                          double* gptq_loss, int* status_dev,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * GPTQ for several layers that share their input (Section 3.3 and Appendix B give the per-layer
+ * flow: the dimension is chosen with RTN, then GPTQ runs in it; in a transformer block q, k, v
+ * (and gate, up) read the same activations, hence the same H and U).  The layers' working rows are
+ * stacked, so one chain of 128-column steps serves all of them: the sequential depth of the
+ * method is paid once instead of once per layer, and the device is filled by 3-4 times the rows.
+ * Every layer is quantized exactly as adadim_quantize_gptq would quantize it alone.
+ *   layers     host array of n_layers descriptors (read during the call only).  Per layer:
+ *                W, out, ldw      the weight [out][in], element type wdtype (shared), out % 128 == 0
+ *                q_oc, q_ic       outputs; both are required for ADADIM_DIM_BOTH and
+ *                                 ADADIM_DIM_CHOSEN, the one named by dim otherwise
+ *                dim              ADADIM_DIM_OC, _IC, _BOTH, or ADADIM_DIM_CHOSEN: the dimension is read
+ *                                 on the device from *chosen when the kernels run (for example the
+ *                                 word adadim_score_select wrote for this layer's RTN results), so
+ *                                 the paper's flow needs no host round trip between its two halves;
+ *                                 only the chosen tensor is written
+ *                chosen           device int (adadim_dim), used with ADADIM_DIM_CHOSEN
+ *                gptq_loss        optional device double[2]: element [dim] receives 1/2 sum e^2
+ *   A layer in both dimensions counts as two working copies; at most ADADIM_MAX_BATCHED_LAYERS
+ *   copies per call.  workspace: adadim_workspace_bytes(ADADIM_WS_GPTQ_ROWS, rows, in, ..) with
+ *   rows the total of the copies' out.  Other arguments as adadim_quantize_gptq.
+ */
+#define ADADIM_MAX_BATCHED_LAYERS 16
+typedef struct {
+  const void* W;
+  int64_t out;
+  int64_t ldw;
+  const adadim_qtensor* q_oc;
+  const adadim_qtensor* q_ic;
+  int dim;
+  const int* chosen;
+  double* gptq_loss;
+} adadim_gptq_layer;
+ADADIM_API int adadim_quantize_gptq_batched(const adadim_gptq_layer* layers, int n_layers, int wdtype, int64_t in,
+                         const float* H, const double* U, int bits, int group,
+                         double percdamp, int blocksize, int* status_dev,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*

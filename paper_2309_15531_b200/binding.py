@@ -16,8 +16,8 @@ import torch
 
 OK = 0
 F32, F16, BF16 = 0, 1, 2
-DIM_OC, DIM_IC, DIM_BOTH = 0, 1, 2
-WS_HESSIAN, WS_GPTQ, WS_SCORE, WS_FACTOR = 0, 1, 2, 3
+DIM_OC, DIM_IC, DIM_BOTH, DIM_CHOSEN = 0, 1, 2, 3
+WS_HESSIAN, WS_GPTQ, WS_SCORE, WS_FACTOR, WS_GPTQ_ROWS = 0, 1, 2, 3, 4
 DIM_NAMES = {DIM_OC: "oc", DIM_IC: "ic"}
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadadim.so")
@@ -32,6 +32,11 @@ class AdadimError(RuntimeError):
 
 class QTensorC(C.Structure):
     _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p), ("zeros", C.c_void_p)]
+
+
+class GptqLayerC(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("out", C.c_int64), ("ldw", C.c_int64), ("q_oc", C.POINTER(QTensorC)),
+                ("q_ic", C.POINTER(QTensorC)), ("dim", C.c_int), ("chosen", C.c_void_p), ("gptq_loss", C.c_void_p)]
 
 
 def lib():
@@ -57,6 +62,9 @@ def lib():
         L.adadim_quantize_gptq.restype = C.c_int
         L.adadim_quantize_gptq.argtypes = [vp, C.c_int, i64, i64, i64, vp, vp, C.c_int, C.c_int, C.c_int, C.c_double,
                                            C.c_int, qp, qp, vp, vp, vp, sz, vp]
+        L.adadim_quantize_gptq_batched.restype = C.c_int
+        L.adadim_quantize_gptq_batched.argtypes = [C.POINTER(GptqLayerC), C.c_int, C.c_int, i64, vp, vp, C.c_int,
+                                                   C.c_int, C.c_double, C.c_int, vp, vp, sz, vp]
         L.adadim_quantize_gptq_reordered.restype = C.c_int
         L.adadim_quantize_gptq_reordered.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, C.c_int,
                                                      C.c_double, C.c_int, qp, qp, vp, vp, vp, vp, sz, vp]
@@ -184,6 +192,46 @@ def quantize_gptq(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, dim: 
                                     workspace.data_ptr(), workspace.numel(), _stream())
     _check(rc, "adadim_quantize_gptq")
     return q_oc, q_ic
+
+
+def quantize_gptq_batched(Ws, H: torch.Tensor, bits: int, group: int, dims, percdamp: float = 0.01,
+                          U: Optional[torch.Tensor] = None, chosen=None, qs=None, losses=None,
+                          status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+    """GPTQ for layers that share H (and U): one call, one chain of column steps for all of them.
+    Ws: list of weights [out_l, in] of one dtype; dims: one of DIM_OC / DIM_IC / DIM_BOTH / DIM_CHOSEN per
+    layer; chosen: per layer a device int32[1] (required for DIM_CHOSEN, e.g. score_select's output);
+    qs: optional list of (q_oc, q_ic) to write into.  Returns the list of (q_oc, q_ic); with DIM_CHOSEN
+    both are allocated and the one named by the device word is written."""
+    n = len(Ws)
+    inp = Ws[0].shape[1]
+    assert all(w.is_cuda and w.stride(1) == 1 and w.shape[1] == inp and w.dtype == Ws[0].dtype for w in Ws)
+    out_qs, keep, arr = [], [], (GptqLayerC * n)()
+    rows = 0
+    for l, W in enumerate(Ws):
+        out, dim = W.shape[0], dims[l]
+        q_oc, q_ic = qs[l] if qs is not None else (None, None)
+        if dim != DIM_IC and q_oc is None:
+            q_oc = QTensor(out, inp, bits, group, DIM_OC, W.device)
+        if dim != DIM_OC and q_ic is None:
+            q_ic = QTensor(out, inp, bits, group, DIM_IC, W.device)
+        coc = q_oc.c() if q_oc is not None else None
+        cic = q_ic.c() if q_ic is not None else None
+        keep.append((coc, cic))
+        arr[l].W, arr[l].out, arr[l].ldw, arr[l].dim = W.data_ptr(), out, W.stride(0), dim
+        arr[l].q_oc = C.pointer(coc) if coc is not None else None
+        arr[l].q_ic = C.pointer(cic) if cic is not None else None
+        arr[l].chosen = chosen[l].data_ptr() if chosen is not None and chosen[l] is not None else None
+        arr[l].gptq_loss = losses[l].data_ptr() if losses is not None and losses[l] is not None else None
+        out_qs.append((q_oc, q_ic))
+        rows += out * (2 if dim == DIM_BOTH else 1)
+    if workspace is None:
+        workspace = _ws(workspace_bytes(WS_GPTQ_ROWS, rows, inp, bits, group), Ws[0].device)
+    rc = lib().adadim_quantize_gptq_batched(arr, n, _DT[Ws[0].dtype], inp, H.data_ptr(),
+                                            U.data_ptr() if U is not None else None, bits, group, percdamp, 128,
+                                            status.data_ptr() if status is not None else None,
+                                            workspace.data_ptr(), workspace.numel(), _stream())
+    _check(rc, "adadim_quantize_gptq_batched")
+    return out_qs
 
 
 def quantize_gptq_reordered(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, dim: int = DIM_BOTH,

@@ -15,10 +15,19 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* status_dev, void* workspace,
                   cudaStream_t st, const int* perm);
-size_t gptq_workspace_bytes(int64_t out, int64_t in);
-int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const double* U,
-                int bits, int group, int dim, double percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
-                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st, bool reorder, int* perm_out);
+size_t gptq_workspace_bytes(int64_t rows, int64_t in);
+struct GptqLayer {
+  const void* W;
+  int64_t out, ldw;
+  const adadim_qtensor* q_oc;
+  const adadim_qtensor* q_ic;
+  int dim;
+  const int* chosen;
+  double* loss;
+};
+int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, const float* H, const double* U,
+                int bits, int group, double percdamp, int* status_dev, void* workspace, cudaStream_t st, bool reorder,
+                int* perm_out);
 
 namespace {
 
@@ -96,7 +105,8 @@ size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int g
   if (out < 0 || in < 0) return 0;
   switch (kind) {
     case ADADIM_WS_HESSIAN: return 0;
-    case ADADIM_WS_GPTQ: return gptq_workspace_bytes(out, in);
+    case ADADIM_WS_GPTQ: return gptq_workspace_bytes(2 * out, in);
+    case ADADIM_WS_GPTQ_ROWS: return gptq_workspace_bytes(out, in);
     case ADADIM_WS_SCORE: return score_workspace_bytes(out, in);
     case ADADIM_WS_FACTOR: return factor_workspace_bytes(in);
     default: return 0;
@@ -177,9 +187,46 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
   const bool oc = dim != ADADIM_DIM_IC, ic = dim != ADADIM_DIM_OC;
   if (oc && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
   if (ic && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
-  if (workspace_bytes < gptq_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
-  return gptq_launch(W, wdtype, out, in, ldw, H, U, bits, group, dim, percdamp, q_oc, q_ic, gptq_loss, status_dev,
-                     workspace, st, false, nullptr);
+  if (workspace_bytes < gptq_workspace_bytes(2 * out, in)) return ADADIM_ERR_WORKSPACE;
+  const GptqLayer layer = {W, out, ldw, q_oc, q_ic, dim, nullptr, gptq_loss};
+  return gptq_launch(&layer, 1, wdtype, in, H, U, bits, group, percdamp, status_dev, workspace, st, false, nullptr);
+}
+
+int adadim_quantize_gptq_batched(const adadim_gptq_layer* layers, int n_layers, int wdtype, int64_t in, const float* H,
+                                 const double* U, int bits, int group, double percdamp, int blocksize, int* status_dev,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int rc = check_quant_params(bits, group, false);
+  if (rc != ADADIM_OK) return rc;
+  if (blocksize != 128) return ADADIM_ERR_PARAM;
+  if (!(percdamp >= 0.0) || !(percdamp < 1e6)) return ADADIM_ERR_PARAM;
+  if (n_layers < 0 || n_layers > ADADIM_MAX_BATCHED_LAYERS || in < 0) return ADADIM_ERR_SHAPE;
+  if (n_layers == 0 || in == 0) return ADADIM_OK;
+  if (layers == nullptr || H == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
+  if (in % 128 != 0) return ADADIM_ERR_SHAPE;
+  if (!aligned16(H) || (U != nullptr && !aligned16(U)) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
+  GptqLayer ls[ADADIM_MAX_BATCHED_LAYERS];
+  int64_t rows = 0;
+  int copies = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const adadim_gptq_layer& y = layers[l];
+    if (y.out <= 0 || y.out % 128 != 0) return ADADIM_ERR_SHAPE;
+    rc = check_weight(y.W, wdtype, y.out, in, y.ldw);
+    if (rc != ADADIM_OK) return rc;
+    if (y.dim != ADADIM_DIM_OC && y.dim != ADADIM_DIM_IC && y.dim != ADADIM_DIM_BOTH && y.dim != ADADIM_DIM_CHOSEN)
+      return ADADIM_ERR_PARAM;
+    if (y.dim == ADADIM_DIM_CHOSEN && y.chosen == nullptr) return ADADIM_ERR_NULL;
+    const bool oc = y.dim != ADADIM_DIM_IC, ic = y.dim != ADADIM_DIM_OC;
+    if (oc && (rc = check_qtensor(y.q_oc)) != ADADIM_OK) return rc;
+    if (ic && (rc = check_qtensor(y.q_ic)) != ADADIM_OK) return rc;
+    const int nd = y.dim == ADADIM_DIM_BOTH ? 2 : 1;
+    copies += nd;
+    rows += nd * y.out;
+    ls[l] = {y.W, y.out, y.ldw, y.q_oc, y.q_ic, y.dim, y.chosen, y.gptq_loss};
+  }
+  if (copies > ADADIM_MAX_BATCHED_LAYERS) return ADADIM_ERR_SHAPE;
+  if (workspace_bytes < gptq_workspace_bytes(rows, in)) return ADADIM_ERR_WORKSPACE;
+  return gptq_launch(ls, n_layers, wdtype, in, H, U, bits, group, percdamp, status_dev, workspace, st, false, nullptr);
 }
 
 int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H,
@@ -203,9 +250,10 @@ int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64
   const bool oc = dim != ADADIM_DIM_IC, ic = dim != ADADIM_DIM_OC;
   if (oc && (rc = check_qtensor(q_oc)) != ADADIM_OK) return rc;
   if (ic && (rc = check_qtensor(q_ic)) != ADADIM_OK) return rc;
-  if (workspace_bytes < gptq_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
-  return gptq_launch(W, wdtype, out, in, ldw, H, nullptr, bits, group, dim, percdamp, q_oc, q_ic, gptq_loss,
-                     status_dev, workspace, st, true, perm_out);
+  if (workspace_bytes < gptq_workspace_bytes(2 * out, in)) return ADADIM_ERR_WORKSPACE;
+  const GptqLayer layer = {W, out, ldw, q_oc, q_ic, dim, nullptr, gptq_loss};
+  return gptq_launch(&layer, 1, wdtype, in, H, nullptr, bits, group, percdamp, status_dev, workspace, st, true,
+                     perm_out);
 }
 
 int adadim_score_select(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, int bits,

@@ -55,7 +55,7 @@ constexpr int kUPacked = u_tile_off(4);              // 10240 doubles
 template <typename T>
 __global__ void __launch_bounds__(256)
 init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const float* __restrict__ H, int ndim,
-            double* __restrict__ Wc) {
+            double* __restrict__ Wc /* first of ndim consecutive copies of this layer */) {
   int64_t e = (static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x) * 8;
   if (e >= out * in) return;
   int64_t o = e / in, i = e % in;
@@ -73,21 +73,33 @@ init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const
   }
 }
 
+// One working copy: one layer under one grouping dimension.  The copies of a call (several layers
+// that share the Hessian, each in one or both dimensions) are stacked along the rows, so that one
+// chain of block kernels and one chain of trailing updates serves them all.
+constexpr int kMaxCopies = 16;
+struct Copy {
+  int64_t slab0;             // first 128-row slab of this copy in the stacked working weights
+  int64_t out;               // rows of the layer
+  adadim_qtensor q[2];       // the layer's per-OC and per-IC outputs (only the one in use is written)
+  uint32_t* codes;           // where codes go instead of q[dim].codes (reordered variant: a temporary stream), or null
+  const int* chosen;         // dim < 0: the grouping dimension is read from this device word
+  double* loss;              // optional device double[2] of the layer: element [dim] receives 1/2 sum e^2
+  const uint2* static_rec;   // per-OC static groups (reordered variant): [out][in/g] records
+                             // {bits of 1/s (0: degenerate group), fp16 s | fp16 z << 16}, else null
+  int dim;                   // ADADIM_DIM_OC, ADADIM_DIM_IC, or -1
+};
 struct BlockArgs {
-  double* Wc;                // [ndim] working weights of [out][in] each, in the tiled layout of wc_index()
+  double* Wc;                // stacked working weights [rows][in] in the tiled layout of wc_index()
   const double* U;           // [in][in]
   int* status_dev;
-  __nv_bfloat16* Ep[3];      // [ndim*out][128] errors as three fixed-point bf16 pieces
-  double* loss_part;         // [ndim][out/128]
-  adadim_qtensor q[2];       // outputs for the dimension(s) in flight
-  int dim_of[2];             // grouping dimension of working copy d
-  int64_t out, in;
+  __nv_bfloat16* Ep[3];      // [rows][128] errors as three fixed-point bf16 pieces
+  double* loss_part;         // [rows / 128]
+  int64_t in;
   int i1;                    // first column of the block
-  // activation reordering (null / unused in the natural order): column i of the working copy is
-  // column perm[i] of W; per-OC parameters are fixed per original group beforehand
+  // activation reordering (null in the natural order): column i of the working copy is column perm[i] of W
   const int* perm;
-  const uint2* static_rec;   // [out][in/g]: {bits of 1/s (0: degenerate group), fp16 s | fp16 z << 16}
-  uint32_t* codes[2];        // where the block kernel writes codes (in working-copy column order)
+  int ncopies;
+  Copy c[kMaxCopies];
 };
 
 // ---- activation reordering (paper Section 2.2, Appendix A.1) ---------------------------------
@@ -270,13 +282,19 @@ block_kernel(const BlockArgs a) {
   __shared__ uint64_t bar[2];
   __shared__ int dead_flag;
 
-  const int d = blockIdx.y;
-  const bool is_ic = a.dim_of[d] == ADADIM_DIM_IC;
-  const adadim_qtensor q = a.q[d];
+  int ci = 0;                                        // the copy this slab belongs to
+  while (ci + 1 < a.ncopies && static_cast<int64_t>(blockIdx.x) >= a.c[ci + 1].slab0) ++ci;
+  const Copy& cp = a.c[ci];
+  const int dim = cp.dim >= 0 ? cp.dim : *cp.chosen;
+  const bool is_ic = dim == ADADIM_DIM_IC;
+  const adadim_qtensor q = cp.q[is_ic ? 1 : 0];
+  uint32_t* const codes = cp.codes != nullptr ? cp.codes : q.codes;
+  const uint2* const static_rec = is_ic ? nullptr : cp.static_rec;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kBlk;
+  const int64_t srow0 = static_cast<int64_t>(blockIdx.x) * kBlk;                 // in the stacked working weights
+  const int64_t row0 = (static_cast<int64_t>(blockIdx.x) - cp.slab0) * kBlk;     // in the layer
   const int64_t row = row0 + tid;
-  const double* Wd = a.Wc + static_cast<int64_t>(d) * a.out * a.in;
+  const double* Wd = a.Wc;
 
   // Staging by bulk copies: one memory latency for the U block and one for the slab.  The kernel
   // may have been scheduled while the launch before it in the stream (the update of this block's
@@ -301,7 +319,7 @@ block_kernel(const BlockArgs a) {
   if (tid < kLaterTiles + kFirstTiles) {
     // tile tid of the slab: 4 tile rows x 8 tile columns; the first two tile columns land in Es
     const int tr = tid >> 3, tc = tid & 7;
-    const double* src = Wd + ((row0 / kWcTileRows + tr) * (a.in / kWcTileCols) + a.i1 / kWcTileCols + tc) * kWcTileElems;
+    const double* src = Wd + ((srow0 / kWcTileRows + tr) * (a.in / kWcTileCols) + a.i1 / kWcTileCols + tc) * kWcTileElems;
     double* dst = tc < 2 ? Es + (tr * 2 + tc) * kWcTileElems : Wt + (tr * (kLater / kWcTileCols) + tc - 2) * kWcTileElems;
     ptx::bulk_load(dst, src, kWcTileElems * sizeof(double), &bar[1]);
   }
@@ -356,17 +374,17 @@ block_kernel(const BlockArgs a) {
         *reinterpret_cast<float4*>(Wt + later_at(tid, cbase - kSub + 2 * k)) = ef[k];
     }
     uint2 srec[kSub];                                // static per-OC records of these 32 columns
-    if (!is_ic && a.static_rec != nullptr) {
+    if (static_rec != nullptr) {
 #pragma unroll
       for (int k = 0; k < kSub; ++k)
-        srec[k] = a.static_rec[row * (a.in / G) + a.perm[a.i1 + cbase + k] / G];
+        srec[k] = static_rec[row * (a.in / G) + a.perm[a.i1 + cbase + k] / G];
     }
 
 #pragma unroll
     for (int ii = 0; ii < kSub; ++ii) {
       const int i = cbase + ii;                      // column inside the block
       const float w32 = static_cast<float>(w[ii]);   // the weight as it stands, rounded once: what is quantized
-      if (!is_ic && a.static_rec != nullptr) {       // per-OC, static groups: parameters fixed beforehand
+      if (static_rec != nullptr) {                   // per-OC, static groups: parameters fixed beforehand
         const uint2 rec = srec[ii];
         gp.rcp = __uint_as_float(rec.x);
         gp.s = __half2float(__ushort_as_half(static_cast<unsigned short>(rec.y & 0xffffu)));
@@ -426,7 +444,7 @@ block_kernel(const BlockArgs a) {
       for (int jj = ii + 1; jj < kSub; ++jj) w[jj] = fma(-e, urow[jj], w[jj]);
     }
     // codes of these 32 columns: BITS whole words of this row's bitstream
-    uint32_t* cdst = a.codes[d] + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
+    uint32_t* cdst = codes + row * (a.in * BITS / 32) + static_cast<int64_t>(a.i1 + cbase) * BITS / 32;
 #pragma unroll
     for (int k = 0; k < BITS; ++k) cdst[k] = cw[k];
     // lazy update of the block's later columns with this sub-block's 32 errors, as a small
@@ -452,7 +470,7 @@ block_kernel(const BlockArgs a) {
     gridr[tid] = __int_as_float((ex - 7) << 23);     // grid of this row
   }
   __syncthreads();
-  const int64_t ebase = (static_cast<int64_t>(d) * a.out + row0) * kBlk;
+  const int64_t ebase = srow0 * kBlk;
   // thread tid takes column tid of every row r (e = 128 r + tid): a warp stores 64 contiguous bytes.
   // Column tid = 32 j + k: float k of the 16 slots that hold sub-block j's errors.
   const int eslot = (warp < 3 ? kSub * warp : kLater - kSub / 2) + (lane >> 1);
@@ -483,18 +501,18 @@ block_kernel(const BlockArgs a) {
   for (int m = 16; m > 0; m >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, m);
   if (lane == 0) lred[warp] = loss;
   __syncthreads();
-  if (tid == 0) a.loss_part[static_cast<int64_t>(d) * (a.out / kBlk) + blockIdx.x] += (lred[0] + lred[1]) + (lred[2] + lred[3]);
+  if (tid == 0) a.loss_part[blockIdx.x] += (lred[0] + lred[1]) + (lred[2] + lred[3]);
 }
 
-__global__ void loss_kernel(const double* __restrict__ part, int ndim, int slabs, BlockArgs a, double* loss_out) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
-    loss_out[0] = 0.0; loss_out[1] = 0.0;
-    for (int d = 0; d < ndim; ++d) {
-      double s = 0.0;
-      for (int k = 0; k < slabs; ++k) s += part[d * slabs + k];
-      loss_out[a.dim_of[d]] = 0.5 * s;
-    }
-  }
+// 1/2 sum e^2 of every copy into its layer's loss[dim], the slabs' partial sums in a fixed order.
+__global__ void loss_kernel(const BlockArgs a) {
+  const int ci = threadIdx.x;
+  if (ci >= a.ncopies || a.c[ci].loss == nullptr) return;
+  const Copy& cp = a.c[ci];
+  const int dim = cp.dim >= 0 ? cp.dim : *cp.chosen;
+  double s = 0.0;
+  for (int64_t k = 0; k < cp.out / kBlk; ++k) s += a.loss_part[cp.slab0 + k];
+  cp.loss[dim == ADADIM_DIM_IC ? 1 : 0] = 0.5 * s;
 }
 
 constexpr size_t block_smem_bytes() {
@@ -503,13 +521,13 @@ constexpr size_t block_smem_bytes() {
 }
 
 template <int BITS, int G>
-int block_launch(const BlockArgs& a, int slabs, int ndim, cudaStream_t st) {
+int block_launch(const BlockArgs& a, int slabs, cudaStream_t st) {
   ADADIM_CUDA_TRY(cudaFuncSetAttribute(block_kernel<BITS, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(block_smem_bytes())));
   // launched so that it may be scheduled while the kernel before it in the stream finishes
   // (it waits for that kernel itself, after staging what does not depend on it)
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(slabs, ndim);
+  cfg.gridDim = dim3(slabs);
   cfg.blockDim = dim3(kBlk);
   cfg.dynamicSmemBytes = block_smem_bytes();
   cfg.stream = st;
@@ -524,45 +542,76 @@ int block_launch(const BlockArgs& a, int slabs, int ndim, cudaStream_t st) {
 
 struct GptqLayout {
   size_t wc_off, err_off, err_piece, loss_off, up_off, up_piece, u_off, factor_off;
-  size_t perm_off, rank_off, rec_off, tmp_off, tmp_piece, total;     // used by the reordered variant only
+  size_t perm_off, rank_off, rec_off, tmp_off, total;      // the last four: the reordered variant only
 };
-GptqLayout gptq_layout(int64_t out, int64_t in) {
+// rows: all working copies stacked (a layer quantized in both dimensions counts twice)
+GptqLayout gptq_layout(int64_t rows, int64_t in) {
   GptqLayout L;
   size_t off = 0;
-  L.wc_off = off;     off += round_up(static_cast<size_t>(2) * out * in * 8, 256);
-  L.err_piece = round_up(static_cast<size_t>(2) * 2 * out * kBlk * 2, 1024);      // two alternating sets
+  L.wc_off = off;     off += round_up(static_cast<size_t>(rows) * in * 8, 256);
+  L.err_piece = round_up(static_cast<size_t>(2) * rows * kBlk * 2, 1024);         // two alternating sets
   L.err_off = off;    off += 3 * L.err_piece;
   L.up_piece = round_up(static_cast<size_t>(in) * in * 2, 1024);
   L.up_off = off;     off += 3 * L.up_piece;
-  L.loss_off = off;   off += round_up(static_cast<size_t>(2) * (out / kBlk + 1) * 8, 256);
+  L.loss_off = off;   off += round_up(static_cast<size_t>(rows / kBlk + 2) * 8, 256);
   L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 8, 256);
   L.factor_off = off; off += factor_workspace_bytes(in);
   L.perm_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
   L.rank_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
-  L.rec_off = off;    off += round_up(static_cast<size_t>(out) * (in / 32) * 8, 256);     // g >= 32
-  L.tmp_piece = round_up(static_cast<size_t>(out) * in / 2, 256);                          // bits <= 4
-  L.tmp_off = off;    off += 2 * L.tmp_piece;
+  L.rec_off = off;    off += round_up(static_cast<size_t>(rows) * (in / 32) * 8, 256);    // g >= 32
+  L.tmp_off = off;    off += round_up(static_cast<size_t>(rows) * in / 2, 256);           // bits <= 4
   L.total = off;
   return L;
 }
 
 template <int BITS>
-int block_launch_g(const BlockArgs& a, int group, int slabs, int ndim, cudaStream_t st) {
-  return group == 128 ? block_launch<BITS, 128>(a, slabs, ndim, st)
-       : group == 64  ? block_launch<BITS, 64>(a, slabs, ndim, st)
-                      : block_launch<BITS, 32>(a, slabs, ndim, st);
+int block_launch_g(const BlockArgs& a, int group, int slabs, cudaStream_t st) {
+  return group == 128 ? block_launch<BITS, 128>(a, slabs, st)
+       : group == 64  ? block_launch<BITS, 64>(a, slabs, st)
+                      : block_launch<BITS, 32>(a, slabs, st);
 }
 
 }  // namespace
 
-size_t gptq_workspace_bytes(int64_t out, int64_t in) { return gptq_layout(out, in).total; }
+size_t gptq_workspace_bytes(int64_t rows, int64_t in) { return gptq_layout(rows, in).total; }
 
-int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, const double* U_in,
-                int bits, int group, int dim, double percdamp, const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
-                double* gptq_loss, int* status_dev, void* workspace, cudaStream_t st, bool reorder, int* perm_out) {
-  GptqLayout L = gptq_layout(out, in);
-  uint8_t* ws = static_cast<uint8_t*>(workspace);
+// One layer of a call, as the launcher sees it.
+struct GptqLayer {
+  const void* W;
+  int64_t out, ldw;
+  const adadim_qtensor* q_oc;
+  const adadim_qtensor* q_ic;
+  int dim;                   // ADADIM_DIM_OC / IC / BOTH / CHOSEN
+  const int* chosen;         // device word, for ADADIM_DIM_CHOSEN
+  double* loss;              // optional device double[2]
+};
+
+int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, const float* H, const double* U_in,
+                int bits, int group, double percdamp, int* status_dev, void* workspace, cudaStream_t st, bool reorder,
+                int* perm_out) {
+  // the working copies, stacked in layer order
   BlockArgs a = {};
+  int64_t rows = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const GptqLayer& y = layers[l];
+    const int dims[2] = {y.dim == ADADIM_DIM_BOTH ? ADADIM_DIM_OC : y.dim == ADADIM_DIM_CHOSEN ? -1 : y.dim,
+                         ADADIM_DIM_IC};
+    const int nd = y.dim == ADADIM_DIM_BOTH ? 2 : 1;
+    for (int d = 0; d < nd; ++d) {
+      if (a.ncopies == kMaxCopies) return ADADIM_ERR_PARAM;
+      Copy& c = a.c[a.ncopies++];
+      c.slab0 = rows / kBlk;
+      c.out = y.out;
+      if (y.q_oc != nullptr) c.q[0] = *y.q_oc;
+      if (y.q_ic != nullptr) c.q[1] = *y.q_ic;
+      c.dim = dims[d];
+      c.chosen = y.chosen;
+      c.loss = y.loss;
+      rows += y.out;
+    }
+  }
+  GptqLayout L = gptq_layout(rows, in);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
   a.Wc = reinterpret_cast<double*>(ws + L.wc_off);
   a.status_dev = status_dev;
   const __nv_bfloat16* ep[3];
@@ -573,34 +622,31 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
     up[k] = reinterpret_cast<__nv_bfloat16*>(ws + L.up_off + k * L.up_piece);
   }
   a.loss_part = reinterpret_cast<double*>(ws + L.loss_off);
-  a.out = out;
   a.in = in;
-  int ndim = 0;
-  if (dim == ADADIM_DIM_OC || dim == ADADIM_DIM_BOTH) { a.q[ndim] = *q_oc; a.dim_of[ndim] = ADADIM_DIM_OC; ++ndim; }
-  if (dim == ADADIM_DIM_IC || dim == ADADIM_DIM_BOTH) { a.q[ndim] = *q_ic; a.dim_of[ndim] = ADADIM_DIM_IC; ++ndim; }
 
   int* perm = nullptr;
   int* rank = nullptr;
-  for (int d = 0; d < ndim; ++d) a.codes[d] = a.q[d].codes;
-  if (reorder) {
+  if (reorder) {                                     // one layer, checked by the caller
+    const GptqLayer& y = layers[0];
     perm = reinterpret_cast<int*>(ws + L.perm_off);
     rank = reinterpret_cast<int*>(ws + L.rank_off);
     order_kernel<<<static_cast<unsigned>((in + 255) / 256), 256, 0, st>>>(H, in, perm, rank);
     if (perm_out != nullptr)
       ADADIM_CUDA_TRY(cudaMemcpyAsync(perm_out, perm, static_cast<size_t>(in) * 4, cudaMemcpyDeviceToDevice, st));
     a.perm = perm;
-    for (int d = 0; d < ndim; ++d) a.codes[d] = reinterpret_cast<uint32_t*>(ws + L.tmp_off + d * L.tmp_piece);
-    if (a.dim_of[0] == ADADIM_DIM_OC) {              // static groups for the per-OC copy (always copy 0)
+    for (int d = 0; d < a.ncopies; ++d)
+      a.c[d].codes = reinterpret_cast<uint32_t*>(ws + L.tmp_off + static_cast<size_t>(d) * round_up(static_cast<size_t>(y.out) * in / 2, 256) );
+    if (a.c[0].dim == ADADIM_DIM_OC) {               // static groups for the per-OC copy (always copy 0)
       uint2* rec = reinterpret_cast<uint2*>(ws + L.rec_off);
-      const unsigned sb = static_cast<unsigned>((out * (in / group) + 255) / 256);
+      const unsigned sb = static_cast<unsigned>((y.out * (in / group) + 255) / 256);
       if (wdtype == ADADIM_F16) {
-        if (bits == 3) static_params_kernel<__half, 3><<<sb, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, group, a.q[0], rec);
-        else static_params_kernel<__half, 4><<<sb, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, group, a.q[0], rec);
+        if (bits == 3) static_params_kernel<__half, 3><<<sb, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
+        else static_params_kernel<__half, 4><<<sb, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
       } else {
-        if (bits == 3) static_params_kernel<float, 3><<<sb, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, group, a.q[0], rec);
-        else static_params_kernel<float, 4><<<sb, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, group, a.q[0], rec);
+        if (bits == 3) static_params_kernel<float, 3><<<sb, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
+        else static_params_kernel<float, 4><<<sb, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
       }
-      a.static_rec = rec;
+      a.c[0].static_rec = rec;
     }
   }
 
@@ -616,20 +662,29 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
                           const_cast<__nv_bfloat16*>(up[2]), st);
   if (rc0 != ADADIM_OK) return rc0;
 
-  if (reorder) {
-    const unsigned pb = static_cast<unsigned>((out * in + 255) / 256);
-    if (wdtype == ADADIM_F16) init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, perm, ndim, a.Wc);
-    else init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, H, perm, ndim, a.Wc);
-  } else {
-    const unsigned ib = static_cast<unsigned>((out * in / 8 + 255) / 256);
-    if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(W), out, in, ldw, H, ndim, a.Wc);
-    else init_kernel<<<ib, 256, 0, st>>>(static_cast<const float*>(W), out, in, ldw, H, ndim, a.Wc);
+  {
+    int ci = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      const GptqLayer& y = layers[l];
+      const int nd = y.dim == ADADIM_DIM_BOTH ? 2 : 1;
+      double* dst = a.Wc + a.c[ci].slab0 * kBlk * in;
+      if (reorder) {
+        const unsigned pb = static_cast<unsigned>((y.out * in + 255) / 256);
+        if (wdtype == ADADIM_F16) init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, H, perm, nd, dst);
+        else init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, H, perm, nd, dst);
+      } else {
+        const unsigned ib = static_cast<unsigned>((y.out * in / 8 + 255) / 256);
+        if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, H, nd, dst);
+        else init_kernel<<<ib, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, H, nd, dst);
+      }
+      ci += nd;
+    }
   }
-  ADADIM_CUDA_TRY(cudaMemsetAsync(a.loss_part, 0, static_cast<size_t>(2) * (out / kBlk + 1) * 8, st));
+  const int slabs = static_cast<int>(rows / kBlk);
+  ADADIM_CUDA_TRY(cudaMemsetAsync(a.loss_part, 0, static_cast<size_t>(slabs + 2) * 8, st));
 
-  const int slabs = static_cast<int>(out / kBlk);
   TrailPlan plan;
-  rc0 = trail_plan(&plan, a.Wc, static_cast<int64_t>(ndim) * out, in, ep, up);
+  rc0 = trail_plan(&plan, a.Wc, rows, in, ep, up);
   if (rc0 != ADADIM_OK) return rc0;
   // Block b+1 only needs its own 128 columns from block b's trailing update.  That part runs on a
   // high-priority stream together with the block kernels; the rest of each trailing update runs
@@ -642,18 +697,16 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
     if (rc0 != ADADIM_OK) return rc0;
     cudaStream_t chain = fs.chain, side = fs.side;
     cudaEvent_t ev_block = fs.ev_a, ev_rest = fs.ev_b;
-    const int64_t rows_total = static_cast<int64_t>(ndim) * out;
     // the side-stream launches get the SMs that the block kernel leaves free (finer CTAs were
     // measured slower: every CTA reloads its 96 KB of error pieces and refills the pipeline)
-    const int free_sms = plan.sm_count - slabs * ndim;
-    const int64_t mblocks = rows_total / kBlk;
-    const int rest_split = free_sms >= mblocks ? static_cast<int>(free_sms / mblocks) : 1;
+    const int free_sms = plan.sm_count - slabs % plan.sm_count;
+    const int rest_split = free_sms >= slabs ? free_sms / slabs : 1;
     __nv_bfloat16* ep_base[3] = {a.Ep[0], a.Ep[1], a.Ep[2]};
     bool rest_pending = false;
     for (int i1 = 0; i1 < in; i1 += kBlk) {
       a.i1 = i1;
-      for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows_total * kBlk;
-      int rc = bits == 3 ? block_launch_g<3>(a, group, slabs, ndim, chain) : block_launch_g<4>(a, group, slabs, ndim, chain);
+      for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows * kBlk;
+      int rc = bits == 3 ? block_launch_g<3>(a, group, slabs, chain) : block_launch_g<4>(a, group, slabs, chain);
       if (rc != ADADIM_OK) return rc;
       const int tiles_after = static_cast<int>((in - i1 - kBlk) / kBlk);
       if (tiles_after > 0) {
@@ -678,13 +731,15 @@ int gptq_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw,
     if (rc0 != ADADIM_OK) return rc0;
   }
   if (reorder) {
+    const int64_t out = layers[0].out;
     const unsigned ub = static_cast<unsigned>((out * (in / 32) + 255) / 256);
-    for (int d = 0; d < ndim; ++d) {
-      if (bits == 3) unpermute_codes_kernel<3><<<ub, 256, 0, st>>>(a.codes[d], rank, out, in, a.q[d].codes);
-      else unpermute_codes_kernel<4><<<ub, 256, 0, st>>>(a.codes[d], rank, out, in, a.q[d].codes);
+    for (int d = 0; d < a.ncopies; ++d) {
+      const adadim_qtensor& q = a.c[d].q[a.c[d].dim == ADADIM_DIM_IC ? 1 : 0];
+      if (bits == 3) unpermute_codes_kernel<3><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
+      else unpermute_codes_kernel<4><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
     }
   }
-  if (gptq_loss != nullptr) loss_kernel<<<1, 32, 0, st>>>(a.loss_part, ndim, slabs, a, gptq_loss);
+  loss_kernel<<<1, 32, 0, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 

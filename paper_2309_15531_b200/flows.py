@@ -47,3 +47,58 @@ def gptq_both(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, percdamp:
     q_oc, q_ic = B.quantize_gptq(W, H, bits, group, B.DIM_BOTH, percdamp, U=U, status=status)
     err, chosen = B.score_select(W, H, bits, group, q_oc, q_ic, status=status)
     return int(chosen.item()), err, (q_oc, q_ic)
+
+
+def block_gptq_ada(layers, bits: int, group: int, percdamp: float = 0.01, status: Optional[torch.Tensor] = None,
+                   max_stacked_rows: int = 148 * 128):
+    """The paper's flow (RTN in both dimensions -> score -> select -> GPTQ in the chosen dimension)
+    for the layers of a transformer block, without a host round trip between the two halves.
+
+    layers: list of (name, W, X) with X the calibration activations of that layer's input; layers that
+    are given the SAME X tensor share one Hessian and one factor, and their GPTQ runs stacked in one
+    batched call (at most max_stacked_rows working rows per call: one 128-row slab per SM).  The
+    Hessian and the factor of an input are computed on a second stream while RTN and scoring of that
+    input's layers wait only for the Hessian.
+    Returns {name: (chosen device int32[1], RTN errors device float64[2], (q_oc, q_ic))}: of the two
+    GPTQ tensors only the one named by `chosen` holds the result.
+    """
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    groups = {}
+    for name, W, X in layers:
+        groups.setdefault(id(X), (X, []))[1].append((name, W))
+    result = {}
+    for X, members in groups.values():
+        inp = X.shape[1]
+        H = torch.zeros(inp, inp, device=X.device)
+        B.hessian_accumulate(X, H, status)
+        h_ready = torch.cuda.Event()
+        h_ready.record(main)
+        with torch.cuda.stream(side):                   # the factor needs H only; scoring below runs beside it
+            side.wait_event(h_ready)
+            U = B.cholesky_inverse_factor(H, percdamp, status)
+            u_ready = torch.cuda.Event()
+            u_ready.record(side)
+        chosen, errs = {}, {}
+        for name, W in members:
+            q_oc, q_ic = B.quantize_rtn(W, bits, group, B.DIM_BOTH)
+            errs[name], chosen[name] = B.score_select(W, H, bits, group, q_oc, q_ic, status=status)
+        main.wait_event(u_ready)
+        U.record_stream(main)
+        batch, rows = [], 0
+        def flush():
+            nonlocal batch, rows
+            if not batch:
+                return
+            qs = B.quantize_gptq_batched([W for _, W in batch], H, bits, group, [B.DIM_CHOSEN] * len(batch), percdamp,
+                                         U=U, chosen=[chosen[n] for n, _ in batch], status=status)
+            for (n, _), q in zip(batch, qs):
+                result[n] = (chosen[n], errs[n], q)
+            batch, rows = [], 0
+        for name, W in members:
+            if batch and (rows + W.shape[0] > max_stacked_rows or len(batch) == 16):
+                flush()
+            batch.append((name, W))
+            rows += W.shape[0]
+        flush()
+    return result
