@@ -583,8 +583,9 @@ def run_config(args):
                       "weights_per_s": weights_total / (flow_ms * 1e-3),
                       "weights_per_s_without_hessians": weights_total / ((flow_ms - hess_ms) * 1e-3),
                       "same_choices_as_layer_by_layer": bool(same),
-                      "how": "flows.block_gptq_ada: q,k,v,o stacked in one batched GPTQ call (128 slabs), gate and up "
-                             "in one each... per max_stacked_rows; no host read-back between RTN selection and GPTQ"}
+                      "how": "flows.block_gptq_ada: layers that share an input share H and U and run GPTQ stacked in batched "
+                             "calls of at most 148 slabs (q,k,v,o together; gate, up, down one call each); the factor runs "
+                             "beside RTN and scoring; no host read-back between RTN selection and GPTQ"}
     # the dominant kernel of these configurations too is the Hessian's tensor-core kernel
     big = max(xspecs, key=lambda xs: xs.inp)
     roofline = dict(shared[f"in={big.inp} ({', '.join(xspecs[big])})"]["rooflines"]["hessian"])

@@ -156,9 +156,10 @@ def quantize_rtn(W: torch.Tensor, bits: int, group: int, dim: int = DIM_BOTH,
 
 
 def cholesky_inverse_factor(H: torch.Tensor, percdamp: float = 0.01, status: Optional[torch.Tensor] = None,
-                            workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+                            workspace: Optional[torch.Tensor] = None, U: Optional[torch.Tensor] = None) -> torch.Tensor:
     n = H.shape[0]
-    U = torch.empty(n, n, dtype=torch.float64, device=H.device)
+    if U is None:
+        U = torch.empty(n, n, dtype=torch.float64, device=H.device)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_FACTOR, 0, n), H.device)
     rc = lib().adadim_cholesky_inverse_factor(H.data_ptr(), n, percdamp, U.data_ptr(),

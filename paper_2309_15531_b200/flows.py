@@ -49,6 +49,17 @@ def gptq_both(W: torch.Tensor, H: torch.Tensor, bits: int, group: int, percdamp:
     return int(chosen.item()), err, (q_oc, q_ic)
 
 
+_SIDE_STREAMS = {}
+
+
+def _side_stream(device) -> torch.cuda.Stream:
+    """One extra stream per device, kept for the life of the process."""
+    key = torch.device(device).index if torch.device(device).index is not None else torch.cuda.current_device()
+    if key not in _SIDE_STREAMS:
+        _SIDE_STREAMS[key] = torch.cuda.Stream(device=key)
+    return _SIDE_STREAMS[key]
+
+
 def block_gptq_ada(layers, bits: int, group: int, percdamp: float = 0.01, status: Optional[torch.Tensor] = None,
                    max_stacked_rows: int = 148 * 128):
     """The paper's flow (RTN in both dimensions -> score -> select -> GPTQ in the chosen dimension)
@@ -63,7 +74,7 @@ def block_gptq_ada(layers, bits: int, group: int, percdamp: float = 0.01, status
     GPTQ tensors only the one named by `chosen` holds the result.
     """
     main = torch.cuda.current_stream()
-    side = torch.cuda.Stream()
+    side = _side_stream(layers[0][1].device)
     groups = {}
     for name, W, X in layers:
         groups.setdefault(id(X), (X, []))[1].append((name, W))
@@ -71,12 +82,16 @@ def block_gptq_ada(layers, bits: int, group: int, percdamp: float = 0.01, status
     for X, members in groups.values():
         inp = X.shape[1]
         H = torch.zeros(inp, inp, device=X.device)
+        # buffers the second stream will use come from this stream's pool: they are handed over and
+        # taken back by events, so the caching allocator can reuse them call after call
+        U = torch.empty(inp, inp, dtype=torch.float64, device=X.device)
+        ws_f = torch.empty(B.workspace_bytes(B.WS_FACTOR, 0, inp), dtype=torch.uint8, device=X.device)
         B.hessian_accumulate(X, H, status)
         h_ready = torch.cuda.Event()
         h_ready.record(main)
         with torch.cuda.stream(side):                   # the factor needs H only; scoring below runs beside it
             side.wait_event(h_ready)
-            U = B.cholesky_inverse_factor(H, percdamp, status)
+            B.cholesky_inverse_factor(H, percdamp, status, ws_f, U)
             u_ready = torch.cuda.Event()
             u_ready.record(side)
         chosen, errs = {}, {}
@@ -84,7 +99,6 @@ def block_gptq_ada(layers, bits: int, group: int, percdamp: float = 0.01, status
             q_oc, q_ic = B.quantize_rtn(W, bits, group, B.DIM_BOTH)
             errs[name], chosen[name] = B.score_select(W, H, bits, group, q_oc, q_ic, status=status)
         main.wait_event(u_ready)
-        U.record_stream(main)
         batch, rows = [], 0
         def flush():
             nonlocal batch, rows
