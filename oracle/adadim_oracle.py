@@ -22,7 +22,9 @@ half-step error bound, on-grid reproduction; Hessian against per-entry
 sums and Freivalds probes; trace form against the explicit layer-output
 form of Eq. 1; GPTQ against H = I (reduces to RTN), the identities
 W - Q = Err U and |Err|^2 = trace(D Hd D^T), an independent
-eliminate-one-coordinate (OBS) formulation, and grid-nearest codes.
+eliminate-one-coordinate (OBS) formulation, and grid-nearest codes; the
+dequantized matrix-vector product against an element-by-element loop, the
+identity per-IC(W) x == (per-OC(W^T))^T x and the quantization error bound.
 Every function here has at least one such pin.
 """
 from __future__ import annotations
@@ -377,3 +379,18 @@ def gptq_both(W, H, bits, group, percdamp=0.01):
     W32 = np.asarray(W).astype(F32)
     err = {d: recon_error_trace(W32, r[d]["Q"], H) for d in ("oc", "ic")}
     return select_dim(err["oc"], err["ic"]), err, r
+
+
+# ---------------------------------------------------------------------------
+# Inference with the quantized weights (Section 4.5, Appendix D: the latency
+# of a matrix-vector product with per-IC quantized weights, fp16 input and
+# output).  What such a kernel computes has a plain definition: y = Q x with
+# Q[o, i] = scale * (code - zero), the group parameters indexed as the
+# grouping dimension says.  Any group size that divides the grouped extent
+# is allowed here (Appendix D goes up to 2048).
+# ---------------------------------------------------------------------------
+
+def dequant_matvec(codes, scales, zeros, group, dim, x):
+    """y[o] = sum_i scale * (code[o, i] - zero) * x[i] in binary64 (x, scales, zeros as given)."""
+    Q = dequantize(codes, scales, zeros, group, dim).astype(np.float64)
+    return Q @ np.asarray(x, dtype=np.float64)
