@@ -610,6 +610,72 @@ def run_config(args):
     print(json.dumps(line))
 
 
+# A100-80GB latencies the paper prints for its own per-IC kernel on this workload (Appendix D, Table 10), ms
+PAPER_GEMV_MS = {(4, 128): 0.50477, (4, 256): 0.32926, (4, 512): 0.24570, (4, 2048): 0.20425,
+                 (3, 128): 0.47336, (3, 256): 0.29957, (3, 512): 0.21457, (3, 2048): 0.16735}
+
+
+def run_gemv(args):
+    """The matrix-vector product of Appendix D: weight 4m x m with m = 12288, per-IC groups of 128 ... 2048,
+    INT3 / INT4, fp16 vector in and out.  One step = one product; codes and parameters are seeded random
+    (the product's cost does not depend on their values)."""
+    import torch
+    from paper_2309_15531_b200 import binding as B
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    m = 12288
+    out, inp = 4 * m, m
+    peaks = _peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    g = torch.Generator(device=dev).manual_seed(230915531)
+    x = torch.randn(inp, device=dev, generator=g).half()
+    y = torch.empty(out, dtype=torch.float16, device=dev)
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.time()
+    rows = {}
+    for bits in (4, 3):
+        codes = torch.randint(-2 ** 31, 2 ** 31 - 1, (out, inp * bits // 32), device=dev, generator=g,
+                              dtype=torch.int64).int()
+        for group in (128, 256, 512, 2048):
+            scales = (torch.rand(out // group, inp, device=dev, generator=g) * 0.01 + 0.001).half()
+            zeros = torch.randint(0, 2 ** bits, (out // group, inp), device=dev, generator=g).half()
+            ws = torch.empty(B.workspace_bytes(B.WS_GEMV, out, inp, bits, group), dtype=torch.uint8, device=dev)
+            for _ in range(max(args.warmup, 3)):
+                B.dequant_gemv(codes, scales, zeros, bits, group, x, y, ws)
+            ts = []
+            for k in range(args.steps):
+                flush.fill_(k & 0xFF)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); B.dequant_gemv(codes, scales, zeros, bits, group, x, y, ws); e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            ms = sum(ts) / len(ts)
+            nbytes = out * inp * bits / 8 + (out // group) * inp * 4 + inp * 2 + out * 2
+            ach = nbytes / (ms * 1e-3) / 1e9
+            rows[f"int{bits} g{group}"] = {"ms": ms, "weights_per_s": out * inp / (ms * 1e-3),
+                                           "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                                        "frac": ach / peaks["hbm_gbs"], "algorithmic_bytes": nbytes},
+                                           "paper_a100_ms": PAPER_GEMV_MS[(bits, group)],
+                                           "paper_a100_ms_over_ours": PAPER_GEMV_MS[(bits, group)] / ms}
+    clocks = sampler.stop(t0, time.time())
+    head = rows["int3 g128"]
+    line = {"metric": "per-IC dequant GEMV latency (4m x m, m = 12288; Appendix D Table 10)", "value": head["ms"], "unit": "ms",
+            "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": head["ms"],
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": head["ms"] / PAPER_GEMV_MS[(3, 128)],
+            "vs_baseline_note": "the paper's number is its own kernel on an A100-80GB: context, not a target",
+            "dtype": "s8 (integer matrix instruction on unpacked codes against a 21-bit fixed-point image of scale * x), fp16 in and out",
+            "data": "synthetic", "config": {"workload": "OPT-175B first FFN layer shape W[49152,12288], INT3 g128 (headline); "
+                                                        "all of Table 10's group sizes and both precisions in `cases`",
+                                            "l2": "flushed between steps by writing a 256 MiB buffer", "replicas": 1},
+            "cases": rows, "roofline": dict(head["roofline"], kernel="gemv_product_kernel<3> (+ gemv_prepare_kernel)", traffic=None),
+            "cpu_baseline": None, "e2e": None, "clocks": clocks, "gpu_launches": 2 * 8 * args.steps}
+    print(json.dumps(line))
+
+
 def lib_factor(B, H, U, st, ws_f):
     """adadim_cholesky_inverse_factor into a preallocated U."""
     rc = B.lib().adadim_cholesky_inverse_factor(H.data_ptr(), H.shape[0], 0.01, U.data_ptr(), st.data_ptr(),
@@ -686,12 +752,14 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="q_proj", choices=["q_proj", "down_proj", "block", "mlp70b"])
+    ap.add_argument("--workload", default="q_proj", choices=["q_proj", "down_proj", "block", "mlp70b", "gemv"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "gemv":
+        run_gemv(args)
     elif args.workload != "q_proj":
         run_config(args)
     else:

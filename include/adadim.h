@@ -66,7 +66,7 @@ typedef enum { ADADIM_DIM_OC = 0, ADADIM_DIM_IC = 1, ADADIM_DIM_BOTH = 2, ADADIM
  * total number of working rows of a batched call (sum over its layers of out, twice for a layer
  * quantized in both dimensions). */
 typedef enum { ADADIM_WS_HESSIAN = 0, ADADIM_WS_GPTQ = 1, ADADIM_WS_SCORE = 2,
-               ADADIM_WS_FACTOR = 3, ADADIM_WS_GPTQ_ROWS = 4 } adadim_ws_kind;
+               ADADIM_WS_FACTOR = 3, ADADIM_WS_GPTQ_ROWS = 4, ADADIM_WS_GEMV = 5 } adadim_ws_kind;
 
 /*
  * One quantized tensor (device pointers, caller-owned).
@@ -277,6 +277,21 @@ ADADIM_API int adadim_score_select_static(const void* W, int wdtype, int64_t out
                                           const adadim_qtensor* q_oc, const adadim_qtensor* q_ic,
                                           double* err, int* chosen, int* status_dev, void* cuda_stream);
 ADADIM_API size_t adadim_static_scratch_bytes(void);
+
+/*
+ * y = Q x with the quantized weights of a per-IC quantized layer (Section 4.5 and Appendix D:
+ * one matrix-vector product of a decoder layer, fp16 vector in, fp16 vector out), consuming the
+ * tensors this library emits as they are:  Q[o,i] = scale[o/g, i] * (code[o,i] - zero[o/g, i]).
+ *   q       codes [out][in*bits/32], scales and zeros [out/group][in]   (dim must be ADADIM_DIM_IC)
+ *   bits    3 or 4;  group any multiple of 16 that divides out (Appendix D measures 128 ... 2048)
+ *   x       fp16 [in], 16-byte aligned;  y  fp16 [out].  in % 128 == 0.
+ *   Within every 128-column block the sums are formed exactly in integers against a 21-bit
+ *   fixed-point image of scale * x; blocks are added in binary32 in column order; the result is
+ *   rounded to fp16 once at the end.
+ *   workspace  adadim_workspace_bytes(ADADIM_WS_GEMV, out, in, bits, group), 256-byte aligned.
+ */
+ADADIM_API int adadim_dequant_gemv(const adadim_qtensor* q, int dim, int64_t out, int64_t in, int bits, int group,
+                        const void* x, void* y, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Helpers. */
 ADADIM_API size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int group);

@@ -17,7 +17,7 @@ import torch
 OK = 0
 F32, F16, BF16 = 0, 1, 2
 DIM_OC, DIM_IC, DIM_BOTH, DIM_CHOSEN = 0, 1, 2, 3
-WS_HESSIAN, WS_GPTQ, WS_SCORE, WS_FACTOR, WS_GPTQ_ROWS = 0, 1, 2, 3, 4
+WS_HESSIAN, WS_GPTQ, WS_SCORE, WS_FACTOR, WS_GPTQ_ROWS, WS_GEMV = 0, 1, 2, 3, 4, 5
 DIM_NAMES = {DIM_OC: "oc", DIM_IC: "ic"}
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadadim.so")
@@ -75,6 +75,8 @@ def lib():
         L.adadim_score_select_static.argtypes = [vp, C.c_int, i64, i64, i64, vp, C.c_int, C.c_int, qp, qp, vp, vp,
                                                  vp, vp]
         L.adadim_static_scratch_bytes.restype = sz
+        L.adadim_dequant_gemv.restype = C.c_int
+        L.adadim_dequant_gemv.argtypes = [qp, C.c_int, i64, i64, C.c_int, C.c_int, vp, vp, vp, sz, vp]
         L.adadim_unpack_codes.restype = C.c_int
         L.adadim_unpack_codes.argtypes = [vp, i64, i64, C.c_int, vp, vp]
         _lib = L
@@ -287,6 +289,23 @@ def score_select(W: torch.Tensor, H: torch.Tensor, bits: int, group: int,
                                    workspace.data_ptr(), workspace.numel(), _stream())
     _check(rc, "adadim_score_select")
     return err, chosen
+
+
+def dequant_gemv(codes: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor, bits: int, group: int,
+                 x: torch.Tensor, y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """y = Q x for a per-IC quantized layer: codes int32 [out, in*bits/32], scales / zeros fp16
+    [out/group, in], x fp16 [in]; returns y fp16 [out]."""
+    out, inp = codes.shape[0], scales.shape[1]
+    assert x.dtype == torch.float16 and x.is_contiguous() and codes.is_contiguous()
+    if y is None:
+        y = torch.empty(out, dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = _ws(workspace_bytes(WS_GEMV, out, inp, bits, group), x.device)
+    qc = QTensorC(codes.data_ptr(), scales.data_ptr(), zeros.data_ptr())
+    rc = lib().adadim_dequant_gemv(C.byref(qc), DIM_IC, out, inp, bits, group, x.data_ptr(), y.data_ptr(),
+                                   workspace.data_ptr(), workspace.numel(), _stream())
+    _check(rc, "adadim_dequant_gemv")
+    return y
 
 
 def static_scratch_bytes() -> int:

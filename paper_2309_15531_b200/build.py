@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libadadim.so")
-SOURCES = ["api.cu", "rtn.cu", "tc_gemm.cu", "score.cu", "cholinv.cu", "gptq.cu", "gptq_tc.cu", "score_static.cu"]
+SOURCES = ["api.cu", "rtn.cu", "tc_gemm.cu", "score.cu", "cholinv.cu", "gptq.cu", "gptq_tc.cu", "score_static.cu", "gemv.cu"]
 HEADERS = ["common.cuh", "umma.cuh", os.path.join("..", "..", "include", "adadim.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

@@ -29,6 +29,10 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
                 int bits, int group, double percdamp, int* status_dev, void* workspace, cudaStream_t st, bool reorder,
                 int* perm_out);
 
+size_t gemv_workspace_bytes(int64_t out, int64_t in, int group);
+int gemv_launch(const adadim_qtensor& q, int64_t out, int64_t in, int bits, int group, const void* x, void* y,
+                void* workspace, cudaStream_t st);
+
 namespace {
 
 int check_weight(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw) {
@@ -101,12 +105,13 @@ const char* adadim_strerror(int status) {
 }
 
 size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int group) {
-  (void)bits; (void)group;
+  (void)bits;
   if (out < 0 || in < 0) return 0;
   switch (kind) {
     case ADADIM_WS_HESSIAN: return 0;
     case ADADIM_WS_GPTQ: return gptq_workspace_bytes(2 * out, in);
     case ADADIM_WS_GPTQ_ROWS: return gptq_workspace_bytes(out, in);
+    case ADADIM_WS_GEMV: return group > 0 ? gemv_workspace_bytes(out, in, group) : 0;
     case ADADIM_WS_SCORE: return score_workspace_bytes(out, in);
     case ADADIM_WS_FACTOR: return factor_workspace_bytes(in);
     default: return 0;
@@ -266,6 +271,22 @@ int adadim_score_select(const void* W, int wdtype, int64_t out, int64_t in, int6
   if (!aligned256(workspace)) return ADADIM_ERR_ALIGN;
   if (workspace_bytes < score_workspace_bytes(out, in)) return ADADIM_ERR_WORKSPACE;
   return score_launch(W, wdtype, out, in, ldw, H, bits, group, q_oc, q_ic, err, chosen, status_dev, workspace, st);
+}
+
+int adadim_dequant_gemv(const adadim_qtensor* q, int dim, int64_t out, int64_t in, int bits, int group, const void* x,
+                        void* y, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (bits != 3 && bits != 4) return ADADIM_ERR_PARAM;
+  if (dim != ADADIM_DIM_IC) return ADADIM_ERR_PARAM;
+  if (group < 16 || group % 16 != 0) return ADADIM_ERR_PARAM;
+  if (out < 0 || in < 0) return ADADIM_ERR_SHAPE;
+  if (out == 0 || in == 0) return ADADIM_OK;
+  if (out % group != 0 || in % 128 != 0) return ADADIM_ERR_SHAPE;
+  int rc = check_qtensor(q);
+  if (rc != ADADIM_OK) return rc;
+  if (x == nullptr || y == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
+  if (!aligned16(x) || !aligned256(workspace) || (reinterpret_cast<uintptr_t>(y) & 1u) != 0) return ADADIM_ERR_ALIGN;
+  if (workspace_bytes < gemv_workspace_bytes(out, in, group)) return ADADIM_ERR_WORKSPACE;
+  return gemv_launch(*q, out, in, bits, group, x, y, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int adadim_unpack_codes(const uint32_t* codes, int64_t out, int64_t in, int bits, uint8_t* dst, void* cuda_stream) {
