@@ -110,7 +110,8 @@ ADADIM_API int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_to
  *     z  = clamp(rint(-lo / s), 0, maxq)
  *     c  = clamp(rint(w / s) + z, 0, maxq)          maxq = 2^bits - 1, rint = ties to even
  *   W      [out][in], wdtype ADADIM_F16 or ADADIM_F32; ldw in elements, 16-byte aligned rows.
- *   bits   3 or 4;  group 32, 64, 128 or 256 (the paper's sweep, Section 4.4, uses 64, 128, 256).
+ *   bits   2, 3, 4 or 8 (INT3 is the paper's headline, INT4 its Appendix; 2 and 8 bound the range);
+ *          group 32, 64, 128 or 256 (the paper's sweep, Section 4.4, uses 64, 128, 256).
  *   dim    ADADIM_DIM_OC (q_oc written), ADADIM_DIM_IC (q_ic written) or ADADIM_DIM_BOTH.
  *   Shape rules: in % 32 == 0; per-OC needs in % group == 0; per-IC needs out % group == 0.
  *   out == 0 or in == 0 is accepted and does nothing.

@@ -47,7 +47,7 @@ int check_weight(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
 // group 256 is accepted by the round-to-nearest quantizer and the scorer; GPTQ works in
 // 128-column blocks on 128-row slabs and takes groups that divide 128
 int check_quant_params(int bits, int group, bool allow_256) {
-  if (bits != 3 && bits != 4) return ADADIM_ERR_PARAM;
+  if (bits != 2 && bits != 3 && bits != 4 && bits != 8) return ADADIM_ERR_PARAM;
   if (group != 32 && group != 64 && group != 128 && !(allow_256 && group == 256)) return ADADIM_ERR_PARAM;
   return ADADIM_OK;
 }
@@ -290,7 +290,7 @@ int adadim_dequant_gemv(const adadim_qtensor* q, int dim, int64_t out, int64_t i
 }
 
 int adadim_unpack_codes(const uint32_t* codes, int64_t out, int64_t in, int bits, uint8_t* dst, void* cuda_stream) {
-  if (bits != 3 && bits != 4) return ADADIM_ERR_PARAM;
+  if (bits != 2 && bits != 3 && bits != 4 && bits != 8) return ADADIM_ERR_PARAM;
   if (out < 0 || in < 0 || in % 32 != 0) return ADADIM_ERR_SHAPE;
   if (out == 0 || in == 0) return ADADIM_OK;
   if (codes == nullptr || dst == nullptr) return ADADIM_ERR_NULL;

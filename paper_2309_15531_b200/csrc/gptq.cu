@@ -559,9 +559,18 @@ GptqLayout gptq_layout(int64_t rows, int64_t in) {
   L.perm_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
   L.rank_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
   L.rec_off = off;    off += round_up(static_cast<size_t>(rows) * (in / 32) * 8, 256);    // g >= 32
-  L.tmp_off = off;    off += round_up(static_cast<size_t>(rows) * in / 2, 256);           // bits <= 4
+  L.tmp_off = off;    off += round_up(static_cast<size_t>(rows) * in, 256);               // bits <= 8
   L.total = off;
   return L;
+}
+
+template <typename T>
+void static_params_launch(const T* W, int64_t out, int64_t in, int64_t ldw, int bits, int group, adadim_qtensor q, uint2* rec,
+                          unsigned blocks, cudaStream_t st) {
+  if (bits == 2) static_params_kernel<T, 2><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, q, rec);
+  else if (bits == 3) static_params_kernel<T, 3><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, q, rec);
+  else if (bits == 4) static_params_kernel<T, 4><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, q, rec);
+  else static_params_kernel<T, 8><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, q, rec);
 }
 
 template <int BITS>
@@ -635,17 +644,12 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
       ADADIM_CUDA_TRY(cudaMemcpyAsync(perm_out, perm, static_cast<size_t>(in) * 4, cudaMemcpyDeviceToDevice, st));
     a.perm = perm;
     for (int d = 0; d < a.ncopies; ++d)
-      a.c[d].codes = reinterpret_cast<uint32_t*>(ws + L.tmp_off + static_cast<size_t>(d) * round_up(static_cast<size_t>(y.out) * in / 2, 256) );
+      a.c[d].codes = reinterpret_cast<uint32_t*>(ws + L.tmp_off + static_cast<size_t>(d) * round_up(static_cast<size_t>(y.out) * in, 256));
     if (a.c[0].dim == ADADIM_DIM_OC) {               // static groups for the per-OC copy (always copy 0)
       uint2* rec = reinterpret_cast<uint2*>(ws + L.rec_off);
       const unsigned sb = static_cast<unsigned>((y.out * (in / group) + 255) / 256);
-      if (wdtype == ADADIM_F16) {
-        if (bits == 3) static_params_kernel<__half, 3><<<sb, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
-        else static_params_kernel<__half, 4><<<sb, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
-      } else {
-        if (bits == 3) static_params_kernel<float, 3><<<sb, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
-        else static_params_kernel<float, 4><<<sb, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, group, a.c[0].q[0], rec);
-      }
+      if (wdtype == ADADIM_F16) static_params_launch(static_cast<const __half*>(y.W), y.out, in, y.ldw, bits, group, a.c[0].q[0], rec, sb, st);
+      else static_params_launch(static_cast<const float*>(y.W), y.out, in, y.ldw, bits, group, a.c[0].q[0], rec, sb, st);
       a.c[0].static_rec = rec;
     }
   }
@@ -706,7 +710,8 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
     for (int i1 = 0; i1 < in; i1 += kBlk) {
       a.i1 = i1;
       for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows * kBlk;
-      int rc = bits == 3 ? block_launch_g<3>(a, group, slabs, chain) : block_launch_g<4>(a, group, slabs, chain);
+      int rc = bits == 2 ? block_launch_g<2>(a, group, slabs, chain) : bits == 3 ? block_launch_g<3>(a, group, slabs, chain)
+             : bits == 4 ? block_launch_g<4>(a, group, slabs, chain) : block_launch_g<8>(a, group, slabs, chain);
       if (rc != ADADIM_OK) return rc;
       const int tiles_after = static_cast<int>((in - i1 - kBlk) / kBlk);
       if (tiles_after > 0) {
@@ -735,8 +740,10 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
     const unsigned ub = static_cast<unsigned>((out * (in / 32) + 255) / 256);
     for (int d = 0; d < a.ncopies; ++d) {
       const adadim_qtensor& q = a.c[d].q[a.c[d].dim == ADADIM_DIM_IC ? 1 : 0];
-      if (bits == 3) unpermute_codes_kernel<3><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
-      else unpermute_codes_kernel<4><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
+      if (bits == 2) unpermute_codes_kernel<2><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
+      else if (bits == 3) unpermute_codes_kernel<3><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
+      else if (bits == 4) unpermute_codes_kernel<4><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
+      else unpermute_codes_kernel<8><<<ub, 256, 0, st>>>(a.c[d].codes, rank, out, in, q.codes);
     }
   }
   loss_kernel<<<1, 32, 0, st>>>(a);

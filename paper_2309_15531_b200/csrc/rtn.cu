@@ -17,32 +17,44 @@ constexpr int kPasses = 8;          // 16 rows per pass
 // rint(q) in the low mantissa bits; code = clamp(bits - bias, 0, maxq) with bias = magic - z is
 // one integer add-min-relu; the codes are packed by multiply-add.  |q| stays far below 2^22
 // here because every weight lies inside its own group's range.
+// The eight codes come back as a 64-bit value in two words; only 8-bit codes use the second one.
 template <int BITS>
-__device__ __forceinline__ uint32_t pack8(const float (&w)[8], const float (&s)[8], const float (&r)[8],
-                                          const int (&nbias)[8]) {
+__device__ __forceinline__ uint2 pack8(const float (&w)[8], const float (&s)[8], const float (&r)[8],
+                                       const int (&nbias)[8]) {
   constexpr int maxq = (1 << BITS) - 1;
-  uint32_t acc = 0;
+  uint32_t acc = 0, acc_hi = 0;
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
     const float t = __fadd_rn(quotient(w[k], s[k], r[k]), kRoundMagic);
     const int c = __viaddmin_s32_relu(__float_as_int(t), nbias[k], maxq);
-    acc = static_cast<uint32_t>(c) * (1u << (BITS * k)) + acc;
+    if (BITS * k < 32) acc = static_cast<uint32_t>(c) * (1u << ((BITS * k) & 31)) + acc;
+    else acc_hi = static_cast<uint32_t>(c) * (1u << ((BITS * k) & 31)) + acc_hi;
   }
-  return acc;
+  return make_uint2(acc, acc_hi);
 }
 
 // Pack eight codes (column order) of `BITS` bits and hand back this thread's share of the
 // row's bitstream.  acc arrives as sum_k(tbits_k << BITS*k) - bias, i.e. the packed value.
 template <int BITS>
-__device__ __forceinline__ void store_codes(uint32_t packed, uint32_t* row_words, int colvec, bool ok) {
-  if (BITS == 4) {
+__device__ __forceinline__ void store_codes(uint2 packed2, uint32_t* row_words, int colvec, bool ok) {
+  const uint32_t packed = packed2.x;
+  if (BITS == 8) {          // 64 bits per thread: two whole words
+    if (ok) *reinterpret_cast<uint2*>(row_words + colvec * 2) = packed2;
+  } else if (BITS == 4) {
     if (ok) row_words[colvec] = packed;
+  } else if (BITS == 2) {   // 16 bits per thread: two threads make a word
+    const uint32_t up = __shfl_down_sync(0xffffffffu, packed, 1);
+    if (ok && (colvec & 1) == 0) row_words[colvec >> 1] = packed | (up << 16);
   } else {  // BITS == 3: 24 bits per thread, four threads make three words
     uint32_t up = __shfl_down_sync(0xffffffffu, packed, 1);
     int k = colvec & 3;
     uint32_t word = (packed >> (8 * k)) | (up << (24 - 8 * k));
     if (ok && k < 3) row_words[(colvec >> 2) * 3 + k] = word;
   }
+}
+template <int BITS>
+__device__ __forceinline__ void store_codes(uint32_t packed, uint32_t* row_words, int colvec, bool ok) {
+  store_codes<BITS>(make_uint2(packed, 0u), row_words, colvec, ok);
 }
 
 template <typename T, int BITS, int G, bool DO_OC, bool DO_IC>
@@ -167,11 +179,11 @@ rtn_tile_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw,
         int nb8[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) { s8[k] = gp.s; r8[k] = gp.rcp; nb8[k] = static_cast<int>(gp.z) - kRoundMagicBits; }
-        const uint32_t acc = pack8<BITS>(w[p], s8, r8, nb8);
+        const uint2 acc = pack8<BITS>(w[p], s8, r8, nb8);
         store_codes<BITS>(acc, qoc.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
       }
       if (DO_IC) {
-        const uint32_t acc = pack8<BITS>(w[p], ic_s, ic_r, ic_nb);
+        const uint2 acc = pack8<BITS>(w[p], ic_s, ic_r, ic_nb);
         store_codes<BITS>(acc, qic.codes + (ok ? row : 0) * words_per_row + c0 * BITS / 32, colvec, ok);
       }
     }
@@ -620,24 +632,34 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ codes, int64_t out, i
 
 }  // namespace
 
+template <typename T>
+void launch_bits(const T* W, int64_t out, int64_t in, int64_t ldw, int bits, int group, int dim,
+                 const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
+  if (group == 256) {
+    if (bits == 2) launch_g256<T, 2>(W, out, in, ldw, dim, qoc, qic, st);
+    else if (bits == 3) launch_g256<T, 3>(W, out, in, ldw, dim, qoc, qic, st);
+    else if (bits == 4) launch_g256<T, 4>(W, out, in, ldw, dim, qoc, qic, st);
+    else launch_g256<T, 8>(W, out, in, ldw, dim, qoc, qic, st);
+  } else {
+    if (bits == 2) launch_group<T, 2>(W, out, in, ldw, group, dim, qoc, qic, st);
+    else if (bits == 3) launch_group<T, 3>(W, out, in, ldw, group, dim, qoc, qic, st);
+    else if (bits == 4) launch_group<T, 4>(W, out, in, ldw, group, dim, qoc, qic, st);
+    else launch_group<T, 8>(W, out, in, ldw, group, dim, qoc, qic, st);
+  }
+}
+
 int rtn_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, int bits, int group, int dim,
                const adadim_qtensor& qoc, const adadim_qtensor& qic, cudaStream_t st) {
-  if (group == 256) {
-    if (wdtype == ADADIM_F16) {
-      if (bits == 3) launch_g256<__half, 3>(static_cast<const __half*>(W), out, in, ldw, dim, qoc, qic, st);
-      else launch_g256<__half, 4>(static_cast<const __half*>(W), out, in, ldw, dim, qoc, qic, st);
-    } else {
-      if (bits == 3) launch_g256<float, 3>(static_cast<const float*>(W), out, in, ldw, dim, qoc, qic, st);
-      else launch_g256<float, 4>(static_cast<const float*>(W), out, in, ldw, dim, qoc, qic, st);
-    }
-    return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
-  }
-  if (wdtype == ADADIM_F16) {
-    if (bits == 3) launch_group_half<3>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
-    else launch_group_half<4>(static_cast<const __half*>(W), out, in, ldw, group, dim, qoc, qic, st);
+  if (wdtype == ADADIM_F16 && group != 256 && bits != 8) {
+    // the register-resident f16x2 kernel; its division-free rounding is proven for |w / s| <= 16 (up to 4 bits)
+    const __half* Wh = static_cast<const __half*>(W);
+    if (bits == 2) launch_group_half<2>(Wh, out, in, ldw, group, dim, qoc, qic, st);
+    else if (bits == 3) launch_group_half<3>(Wh, out, in, ldw, group, dim, qoc, qic, st);
+    else launch_group_half<4>(Wh, out, in, ldw, group, dim, qoc, qic, st);
+  } else if (wdtype == ADADIM_F16) {
+    launch_bits(static_cast<const __half*>(W), out, in, ldw, bits, group, dim, qoc, qic, st);
   } else {
-    if (bits == 3) launch_group<float, 3>(static_cast<const float*>(W), out, in, ldw, group, dim, qoc, qic, st);
-    else launch_group<float, 4>(static_cast<const float*>(W), out, in, ldw, group, dim, qoc, qic, st);
+    launch_bits(static_cast<const float*>(W), out, in, ldw, bits, group, dim, qoc, qic, st);
   }
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
@@ -646,8 +668,10 @@ int unpack_launch(const uint32_t* codes, int64_t out, int64_t in, int bits, uint
   int64_t n = out * (in / 32);
   if (n == 0) return ADADIM_OK;
   unsigned blocks = static_cast<unsigned>((n + 255) / 256);
-  if (bits == 3) unpack_kernel<3><<<blocks, 256, 0, st>>>(codes, out, in, dst);
-  else unpack_kernel<4><<<blocks, 256, 0, st>>>(codes, out, in, dst);
+  if (bits == 2) unpack_kernel<2><<<blocks, 256, 0, st>>>(codes, out, in, dst);
+  else if (bits == 3) unpack_kernel<3><<<blocks, 256, 0, st>>>(codes, out, in, dst);
+  else if (bits == 4) unpack_kernel<4><<<blocks, 256, 0, st>>>(codes, out, in, dst);
+  else unpack_kernel<8><<<blocks, 256, 0, st>>>(codes, out, in, dst);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 

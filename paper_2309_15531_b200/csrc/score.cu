@@ -115,8 +115,10 @@ void diff_launch(const T* W, int64_t out, int64_t in, int64_t ldw, int bits, int
                  __nv_bfloat16* Da, const adadim_qtensor& qb, __nv_bfloat16* Db, cudaStream_t st) {
   const int64_t n = out * (in / 8);
   const unsigned blocks = static_cast<unsigned>((n + 255) / 256);
-  if (bits == 3) diff_kernel<T, 3><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
-  else diff_kernel<T, 4><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
+  if (bits == 2) diff_kernel<T, 2><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
+  else if (bits == 3) diff_kernel<T, 3><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
+  else if (bits == 4) diff_kernel<T, 4><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
+  else diff_kernel<T, 8><<<blocks, 256, 0, st>>>(W, out, in, ldw, group, qa, Da, qb, Db);
 }
 
 struct ScoreLayout {

@@ -85,7 +85,7 @@ def _gptq_case(W, X, bits, group, rows=None):
     return out
 
 
-@pytest.mark.parametrize("bits,group", [(3, 128), (4, 128), (3, 64), (4, 32)])
+@pytest.mark.parametrize("bits,group", [(3, 128), (4, 128), (3, 64), (4, 32), (2, 128), (8, 64), (2, 32), (8, 128)])
 def test_small_layers(bits, group):
     W = I.make_weight(I.WeightSpec(512, 512, "f16", 0.02, 0.001, seed=41), "cuda")
     X = I.make_calib(I.CalibSpec(4096, 512, "bf16", "normal", 3, 50.0, 100.0, seed=42), "cuda")

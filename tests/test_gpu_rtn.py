@@ -33,7 +33,17 @@ def test_small_fp32_layer(bits, group):
     _check_both(W, bits, group)
 
 
-@pytest.mark.parametrize("bits,group,out,inp", [(3, 32, 320, 224), (4, 64, 448, 192), (3, 128, 384, 640)])
+@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("group,dtype", [(32, "f16"), (128, "f16"), (64, "f32"), (256, "f16"), (256, "f32")])
+def test_two_and_eight_bit_codes(bits, group, dtype):
+    """The ends of the precision range (the paper's INT3 / INT4 sit between them): 2-bit codes share a
+    32-bit word sixteen at a time, 8-bit codes fill two words per eight weights."""
+    W = I.make_weight(I.WeightSpec(512, 384 if group != 256 else 512, dtype, 0.02, 0.01, seed=76), "cuda")
+    _check_both(W, bits, group)
+
+
+@pytest.mark.parametrize("bits,group,out,inp", [(3, 32, 320, 224), (4, 64, 448, 192), (3, 128, 384, 640), (2, 32, 320, 224),
+                                                (8, 32, 448, 160)])
 def test_ragged_tiles_fp16(bits, group, out, inp):
     W = I.make_weight(I.WeightSpec(out, inp, "f16", 0.02, 0.01, seed=77), "cuda")
     _check_both(W, bits, group)

@@ -43,7 +43,8 @@ def test_small_fp32_layer():
     _score_case(I.make_weight(wspec, "cuda"), I.make_calib(xspec, "cuda"), 3, 128)
 
 
-@pytest.mark.parametrize("out,inp,bits,group", [(1024, 768, 3, 128), (384, 320, 4, 64), (128, 64, 3, 32)])
+@pytest.mark.parametrize("out,inp,bits,group", [(1024, 768, 3, 128), (384, 320, 4, 64), (128, 64, 3, 32), (256, 256, 2, 64),
+                                                (384, 128, 8, 128)])
 def test_fp16_shapes(out, inp, bits, group):
     W = I.make_weight(I.WeightSpec(out, inp, "f16", 0.02, 0.001, seed=61), "cuda")
     X = I.make_calib(I.CalibSpec(2048, inp, "bf16", "normal", 4, 50.0, 100.0, seed=62), "cuda")
