@@ -151,8 +151,9 @@ ADADIM_API int adadim_cholesky_inverse_factor(const float* H, int64_t in, double
  *   H          [in][in] fp32, required: its diagonal marks the dead columns, and when U == NULL
  *              the factor is computed from it into workspace.
  *   U          optional precomputed adadim_cholesky_inverse_factor of the same H, or NULL.
- *   blocksize  128.  group must divide 128 (32, 64, 128; 256 is refused with ADADIM_ERR_PARAM).
- *              in % 128 == 0, out % 128 == 0.
+ *   blocksize  128.  group 32, 64, 128 or 256.  in % 128 == 0, out % 128 == 0; at group 256 a per-OC
+ *              group spans two column blocks and a per-IC group two 128-row slabs (two CTAs of a
+ *              cluster exchange the column's minimum and maximum), so in % 256 == 0 and out % 256 == 0.
  *   gptq_loss  optional device double[2] (OC, IC): 1/2 * sum of e^2 (only the element of a
  *              dimension that was run is written).
  *   workspace  adadim_workspace_bytes(ADADIM_WS_GPTQ, out, in, bits, group), 256-byte aligned.

@@ -44,8 +44,8 @@ int check_weight(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
   return ADADIM_OK;
 }
 
-// group 256 is accepted by the round-to-nearest quantizer and the scorer; GPTQ works in
-// 128-column blocks on 128-row slabs and takes groups that divide 128
+// every entry point takes groups 32, 64, 128 and 256; at 256 GPTQ needs whole pairs of its 128-row
+// slabs and 128-column blocks (out and in multiples of 256)
 int check_quant_params(int bits, int group, bool allow_256) {
   if (bits != 2 && bits != 3 && bits != 4 && bits != 8) return ADADIM_ERR_PARAM;
   if (group != 32 && group != 64 && group != 128 && !(allow_256 && group == 256)) return ADADIM_ERR_PARAM;
@@ -177,7 +177,7 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
                          const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* gptq_loss, int* status_dev,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group, false);
+  int rc = check_quant_params(bits, group, true);
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
@@ -187,6 +187,7 @@ int adadim_quantize_gptq(const void* W, int wdtype, int64_t out, int64_t in, int
   rc = check_weight(W, wdtype, out, in, ldw);
   if (rc != ADADIM_OK) return rc;
   if (in % 128 != 0 || out % 128 != 0) return ADADIM_ERR_SHAPE;
+  if (group == 256 && (in % 256 != 0 || out % 256 != 0)) return ADADIM_ERR_SHAPE;
   if (H == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
   if (!aligned16(H) || (U != nullptr && !aligned16(U)) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
   const bool oc = dim != ADADIM_DIM_IC, ic = dim != ADADIM_DIM_OC;
@@ -201,21 +202,21 @@ int adadim_quantize_gptq_batched(const adadim_gptq_layer* layers, int n_layers, 
                                  const double* U, int bits, int group, double percdamp, int blocksize, int* status_dev,
                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group, false);
+  int rc = check_quant_params(bits, group, true);
   if (rc != ADADIM_OK) return rc;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
   if (!(percdamp >= 0.0) || !(percdamp < 1e6)) return ADADIM_ERR_PARAM;
   if (n_layers < 0 || n_layers > ADADIM_MAX_BATCHED_LAYERS || in < 0) return ADADIM_ERR_SHAPE;
   if (n_layers == 0 || in == 0) return ADADIM_OK;
   if (layers == nullptr || H == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
-  if (in % 128 != 0) return ADADIM_ERR_SHAPE;
+  if (in % 128 != 0 || (group == 256 && in % 256 != 0)) return ADADIM_ERR_SHAPE;
   if (!aligned16(H) || (U != nullptr && !aligned16(U)) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
   GptqLayer ls[ADADIM_MAX_BATCHED_LAYERS];
   int64_t rows = 0;
   int copies = 0;
   for (int l = 0; l < n_layers; ++l) {
     const adadim_gptq_layer& y = layers[l];
-    if (y.out <= 0 || y.out % 128 != 0) return ADADIM_ERR_SHAPE;
+    if (y.out <= 0 || y.out % 128 != 0 || (group == 256 && y.out % 256 != 0)) return ADADIM_ERR_SHAPE;
     rc = check_weight(y.W, wdtype, y.out, in, y.ldw);
     if (rc != ADADIM_OK) return rc;
     if (y.dim != ADADIM_DIM_OC && y.dim != ADADIM_DIM_IC && y.dim != ADADIM_DIM_BOTH && y.dim != ADADIM_DIM_CHOSEN)
@@ -240,7 +241,7 @@ int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64
                                    int32_t* perm_out, int* status_dev, void* workspace, size_t workspace_bytes,
                                    void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int rc = check_quant_params(bits, group, false);
+  int rc = check_quant_params(bits, group, true);
   if (rc != ADADIM_OK) return rc;
   if (dim != ADADIM_DIM_OC && dim != ADADIM_DIM_IC && dim != ADADIM_DIM_BOTH) return ADADIM_ERR_PARAM;
   if (blocksize != 128) return ADADIM_ERR_PARAM;
@@ -250,6 +251,7 @@ int adadim_quantize_gptq_reordered(const void* W, int wdtype, int64_t out, int64
   rc = check_weight(W, wdtype, out, in, ldw);
   if (rc != ADADIM_OK) return rc;
   if (in % 128 != 0 || out % 128 != 0) return ADADIM_ERR_SHAPE;
+  if (group == 256 && (in % 256 != 0 || out % 256 != 0)) return ADADIM_ERR_SHAPE;
   if (H == nullptr || workspace == nullptr) return ADADIM_ERR_NULL;
   if (!aligned16(H) || !aligned256(workspace)) return ADADIM_ERR_ALIGN;
   const bool oc = dim != ADADIM_DIM_IC, ic = dim != ADADIM_DIM_OC;

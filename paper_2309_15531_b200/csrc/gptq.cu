@@ -94,6 +94,7 @@ struct BlockArgs {
   int* status_dev;
   __nv_bfloat16* Ep[3];      // [rows][128] errors as three fixed-point bf16 pieces
   double* loss_part;         // [rows / 128]
+  float* oc_rcp;             // [rows] g = 256 only: 1 / s of the row's current per-OC group, handed from the group's first block to its second
   int64_t in;
   int i1;                    // first column of the block
   // activation reordering (null in the natural order): column i of the working copy is column perm[i] of W
@@ -268,7 +269,7 @@ __global__ void __launch_bounds__(kBlk, 1)
 block_kernel(const BlockArgs a) {
   constexpr float maxq = static_cast<float>((1 << BITS) - 1);
   constexpr float rcp_maxq = 1.0f / maxq;            // correctly rounded at compile time
-  constexpr int NG = kBlk / G;                       // per-IC groups in the slab
+  constexpr int NG = G >= kBlk ? 1 : kBlk / G;       // per-IC groups in the slab (g = 256: half a group)
   extern __shared__ __align__(128) double smd[];
   double* Wt = smd;                                  // 24 tiles: columns 32..127 of the slab (later_at)
   double* Us = Wt + kLaterTiles * kWcTileElems;      // packed upper block-triangle of the U block
@@ -281,6 +282,7 @@ block_kernel(const BlockArgs a) {
   uint16_t* Zs = Ss + NG * kBlk;                          // [NG][128]
   __shared__ uint64_t bar[2];
   __shared__ int dead_flag;
+  __shared__ float xch[4];                           // g = 256: the neighbouring slab's per-IC minimum and maximum, two slots
 
   int ci = 0;                                        // the copy this slab belongs to
   while (ci + 1 < a.ncopies && static_cast<int64_t>(blockIdx.x) >= a.c[ci + 1].slab0) ++ci;
@@ -390,21 +392,40 @@ block_kernel(const BlockArgs a) {
         gp.s = __half2float(__ushort_as_half(static_cast<unsigned short>(rec.y & 0xffffu)));
         gp.z = __half2float(__ushort_as_half(static_cast<unsigned short>(rec.y >> 16)));
       } else if (!is_ic) {
-        if ((ii % G) == 0 && (cbase % G) == 0) {     // per-OC: parameters at the group's first column
+        if ((ii % G) == 0 && ((a.i1 + cbase) % G) == 0) {     // per-OC: parameters at the group's first column
           float mn = w32, mx = w32;
 #pragma unroll
           for (int k = 1; k < (G < kSub ? G : kSub); ++k) {
             const float v = static_cast<float>(w[ii + k < kSub ? ii + k : kSub - 1]);
             mn = fminf(mn, v); mx = fmaxf(mx, v);
           }
-          for (int k = kSub; k < G; ++k) {           // the group's columns beyond the ones in registers
+          for (int k = kSub; k < (G < kBlk ? G : kBlk); ++k) {    // the group's columns beyond the ones in registers
             const float v = static_cast<float>(Wt[later_at(tid, cbase + k - kSub)]);
             mn = fminf(mn, v); mx = fmaxf(mx, v);
+          }
+          if (G > kBlk) {
+            // g = 256: the group's other 128 columns are the next block's, read where they stand in the
+            // working weights (every update of earlier blocks has reached them: the host orders this
+            // block kernel behind the side stream's launch at a group's first block)
+            const double* nxt = a.Wc + ((srow0 + tid) >> 5) * (a.in >> 4) * kWcTileElems + ((a.i1 + kBlk) >> 4) * kWcTileElems;
+#pragma unroll 4
+            for (int k2 = 0; k2 < kBlk / 2; ++k2) {
+              const double2 t = *reinterpret_cast<const double2*>(nxt + (k2 >> 3) * kWcTileElems + wc_in_tile(lane, 2 * (k2 & 7)));
+              const float v0 = static_cast<float>(t.x), v1 = static_cast<float>(t.y);
+              mn = fminf(mn, fminf(v0, v1)); mx = fmaxf(mx, fmaxf(v0, v1));
+            }
           }
           gp = group_params(mn, mx, maxq, rcp_maxq);
           int64_t idx = row * (a.in / G) + (a.i1 + i) / G;
           q.scales[idx] = __half_as_ushort(__float2half_rn(gp.s));
           q.zeros[idx] = __half_as_ushort(__float2half_rn(gp.z));
+          if (G > kBlk) a.oc_rcp[srow0 + tid] = gp.rcp;
+        } else if (G > kBlk && i == 0) {
+          // g = 256, the group's second block: the parameters its first block took
+          const int64_t idx = row * (a.in / G) + a.i1 / G;
+          gp.s = __half2float(__ushort_as_half(q.scales[idx]));
+          gp.z = __half2float(__ushort_as_half(q.zeros[idx]));
+          gp.rcp = a.oc_rcp[srow0 + tid];
         }
       } else {                                       // per-IC: parameters of this column's g-row groups
         // warp minimum and maximum in one reduction instruction each, on a key that orders
@@ -416,11 +437,27 @@ block_kernel(const BlockArgs a) {
           float* slot = red + (ii & 1) * 8;
           if (lane == 0) { slot[warp * 2] = mn; slot[warp * 2 + 1] = mx; }
           __syncthreads();
-          constexpr int WPG = G / 32;                // warps per group
+          constexpr int WPG = (G < kBlk ? G : kBlk) / 32;     // warps per group (g = 256: all four, half a group)
           const int w0 = (warp / WPG) * WPG;
           mn = slot[w0 * 2]; mx = slot[w0 * 2 + 1];
 #pragma unroll
           for (int k = 1; k < WPG; ++k) { mn = fminf(mn, slot[(w0 + k) * 2]); mx = fmaxf(mx, slot[(w0 + k) * 2 + 1]); }
+        }
+        if (G > kBlk) {
+          // g = 256: a group spans this slab and its neighbour, which the other CTA of the pair (a
+          // cluster of two) holds.  Each writes its minimum and maximum into the other's shared memory;
+          // the cluster barrier orders the writes before the reads.  Slots alternate with the column: a
+          // CTA can reach its write for column ii + 2 only after the other has passed the barrier of
+          // column ii + 1, i.e. after it has read the slot of column ii.
+          float* mine = xch + (ii & 1) * 2;
+          if (tid == 0) {
+            const uint32_t remote = ptx::map_to_cta(ptx::smem_addr(mine), ptx::cluster_ctarank() ^ 1u);
+            ptx::st_cluster_f32(remote, mn);
+            ptx::st_cluster_f32(remote + 4, mx);
+          }
+          ptx::cluster_sync();
+          mn = fminf(mn, mine[0]);
+          mx = fmaxf(mx, mine[1]);
         }
         gp = group_params(mn, mx, maxq, rcp_maxq);
         if ((tid % G) == 0) {
@@ -531,17 +568,24 @@ int block_launch(const BlockArgs& a, int slabs, cudaStream_t st) {
   cfg.blockDim = dim3(kBlk);
   cfg.dynamicSmemBytes = block_smem_bytes();
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (G > kBlk) {                                    // pairs of slabs exchange per-IC statistics: clusters of two CTAs
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   ADADIM_CUDA_TRY(cudaLaunchKernelEx(&cfg, block_kernel<BITS, G>, a));
   return ADADIM_OK;
 }
 
 struct GptqLayout {
-  size_t wc_off, err_off, err_piece, loss_off, up_off, up_piece, u_off, factor_off;
+  size_t wc_off, err_off, err_piece, loss_off, rcp_off, up_off, up_piece, u_off, factor_off;
   size_t perm_off, rank_off, rec_off, tmp_off, total;      // the last four: the reordered variant only
 };
 // rows: all working copies stacked (a layer quantized in both dimensions counts twice)
@@ -554,6 +598,7 @@ GptqLayout gptq_layout(int64_t rows, int64_t in) {
   L.up_piece = round_up(static_cast<size_t>(in) * in * 2, 1024);
   L.up_off = off;     off += 3 * L.up_piece;
   L.loss_off = off;   off += round_up(static_cast<size_t>(rows / kBlk + 2) * 8, 256);
+  L.rcp_off = off;    off += round_up(static_cast<size_t>(rows) * 4, 256);
   L.u_off = off;      off += round_up(static_cast<size_t>(in) * in * 8, 256);
   L.factor_off = off; off += factor_workspace_bytes(in);
   L.perm_off = off;   off += round_up(static_cast<size_t>(in) * 4, 256);
@@ -575,7 +620,8 @@ void static_params_launch(const T* W, int64_t out, int64_t in, int64_t ldw, int 
 
 template <int BITS>
 int block_launch_g(const BlockArgs& a, int group, int slabs, cudaStream_t st) {
-  return group == 128 ? block_launch<BITS, 128>(a, slabs, st)
+  return group == 256 ? block_launch<BITS, 256>(a, slabs, st)
+       : group == 128 ? block_launch<BITS, 128>(a, slabs, st)
        : group == 64  ? block_launch<BITS, 64>(a, slabs, st)
                       : block_launch<BITS, 32>(a, slabs, st);
 }
@@ -631,6 +677,7 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
     up[k] = reinterpret_cast<__nv_bfloat16*>(ws + L.up_off + k * L.up_piece);
   }
   a.loss_part = reinterpret_cast<double*>(ws + L.loss_off);
+  a.oc_rcp = reinterpret_cast<float*>(ws + L.rcp_off);
   a.in = in;
 
   int* perm = nullptr;
@@ -710,6 +757,12 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
     for (int i1 = 0; i1 < in; i1 += kBlk) {
       a.i1 = i1;
       for (int k = 0; k < 3; ++k) a.Ep[k] = ep_base[k] + static_cast<int64_t>((i1 / kBlk) & 1) * rows * kBlk;
+      if (group > kBlk && i1 % group == 0 && rest_pending) {
+        // g = 256: per-OC statistics at a group's first block also read the NEXT block's columns, which
+        // the side stream's launch of the block before last wrote
+        ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
+        rest_pending = false;
+      }
       int rc = bits == 2 ? block_launch_g<2>(a, group, slabs, chain) : bits == 3 ? block_launch_g<3>(a, group, slabs, chain)
              : bits == 4 ? block_launch_g<4>(a, group, slabs, chain) : block_launch_g<8>(a, group, slabs, chain);
       if (rc != ADADIM_OK) return rc;

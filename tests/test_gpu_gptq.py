@@ -92,6 +92,28 @@ def test_small_layers(bits, group):
     _gptq_case(W, X, bits, group)
 
 
+@pytest.mark.parametrize("bits", [3, 4])
+def test_group_256(bits):
+    """The largest group of the paper's sweep (Section 4.4): a per-IC group spans two 128-row slabs
+    (two CTAs exchange minima and maxima per column), a per-OC group two 128-column blocks."""
+    W = I.make_weight(I.WeightSpec(512, 512, "f16", 0.02, 0.001, seed=141), "cuda")
+    X = I.make_calib(I.CalibSpec(4096, 512, "bf16", "normal", 3, 50.0, 100.0, seed=142), "cuda")
+    _gptq_case(W, X, bits, 256)
+
+
+def test_group_256_identity_hessian_reduces_to_rtn_and_skewed_case():
+    W = I.make_weight(I.WeightSpec(256, 512, "f16", 0.02, 0.0, seed=143), "cuda")
+    H = 2.0 * torch.eye(512, device="cuda")
+    q_oc, q_ic = B.quantize_gptq(W, H, 3, 256, B.DIM_BOTH)
+    r_oc, r_ic = B.quantize_rtn(W, 3, 256)
+    torch.cuda.synchronize()
+    for a, b in ((q_oc, r_oc), (q_ic, r_ic)):
+        assert torch.equal(a.codes, b.codes) and torch.equal(a.scales, b.scales) and torch.equal(a.zeros, b.zeros)
+    W = I.make_weight(I.WeightSpec(256, 768, "f16", 0.015, 0.0, seed=144), "cuda")
+    X = I.make_calib(I.CalibSpec(4096, 768, "bf16", "skew", 2, 80.0, 80.0, seed=145), "cuda")
+    _gptq_case(W, X, 4, 256)
+
+
 def test_skewed_activations():
     W = I.make_weight(I.WeightSpec(128, 640, "f16", 0.015, 0.0, seed=43), "cuda")
     X = I.make_calib(I.CalibSpec(4096, 640, "bf16", "skew", 2, 80.0, 80.0, seed=44), "cuda")
@@ -153,6 +175,15 @@ def test_full_size_q_proj_sampled_slabs():
         tr = 0.5 * float(((D @ Hd_t) * D).sum().item())
         print(f"gptq {name}: loss {loss[k].item():.6e}  1/2 trace(D Hd D^T) {tr:.6e}")
         assert loss[k].item() == pytest.approx(tr, rel=1e-3)
+
+
+def test_full_size_q_proj_group_256():
+    """4096 x 4096 at g = 256 on one 256-row group of rows (clusters of two slabs, groups of two blocks)."""
+    wl = I.workload_qproj(n_tokens=16384)
+    wspec, xspec = wl["layers"]["q_proj"]
+    W = I.make_weight(wspec, "cuda")
+    X = I.make_calib(xspec, "cuda")
+    _gptq_case(W, X, 3, 256, rows=slice(1280, 1536))
 
 
 def test_batched_layers_equal_the_single_layer_calls_and_follow_the_device_choice():

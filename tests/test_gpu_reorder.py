@@ -25,7 +25,7 @@ def _run(W, Hn, bits, group, dim=B.DIM_BOTH):
     return q_oc, q_ic, loss.cpu().numpy(), perm.cpu().numpy()
 
 
-@pytest.mark.parametrize("bits,group", [(3, 128), (4, 64), (3, 32), (2, 64), (8, 128)])
+@pytest.mark.parametrize("bits,group", [(3, 128), (4, 64), (3, 32), (2, 64), (8, 128), (3, 256)])
 def test_reordered_small_layers(bits, group):
     W = I.make_weight(I.WeightSpec(512, 512, "f16", 0.02, 0.001, seed=61), "cuda")
     X = I.make_calib(I.CalibSpec(4096, 512, "bf16", "normal", 3, 50.0, 100.0, seed=62), "cuda")

@@ -147,8 +147,11 @@ def test_group_256_selection_flow():
     assert err[0].item() == pytest.approx(ref["oc"], rel=1e-3) and err[1].item() == pytest.approx(ref["ic"], rel=1e-3)
 
 
-def test_gptq_refuses_group_256():
-    W = I.make_weight(I.WeightSpec(256, 256, "f16", 0.02, 0.0, seed=88), "cuda")
-    H = 2.0 * torch.eye(256, device="cuda")
-    with pytest.raises(Exception):
+def test_gptq_group_256_needs_whole_pairs_of_slabs_and_blocks():
+    """GPTQ at g = 256 works on pairs of its 128-row slabs and 128-column blocks: shapes that are
+    multiples of 128 but not of 256 are refused on the host."""
+    H = 2.0 * torch.eye(384, device="cuda")
+    W = I.make_weight(I.WeightSpec(256, 384, "f16", 0.02, 0.0, seed=88), "cuda")
+    with pytest.raises(B.AdadimError) as e:
         B.quantize_gptq(W, H, 3, 256, B.DIM_BOTH)
+    assert e.value.status == 2
