@@ -87,15 +87,18 @@ typedef struct {
 /*
  * Calibration Hessian  H += 2 * X^T X  over one chunk of tokens (Section 4.4: the inverse
  * Hessian GPTQ uses is "formed by activations"; Section 2.2).
- *   X        [n_tokens][in], xdtype ADADIM_BF16 (tcgen05 tensor-core path) or ADADIM_F32.
+ *   X        [n_tokens][in], xdtype ADADIM_BF16 or ADADIM_F32, both on the tcgen05 tensor cores: an
+ *            fp32 chunk is split exactly into three bf16 pieces in the workspace (without a
+ *            workspace of that size a plain multiply-add kernel is used instead).
  *            ldx in elements; X and ldx*sizeof(elem) must be 16-byte aligned.
  *   H        [in][in] fp32, in/out, symmetric on entry: the caller zeroes it before the first
  *            chunk and passes it back unchanged for the next ones.  Both triangles are valid
  *            on return.  in must be a multiple of 8.
  *   n_seen   host pointer, in/out, may be NULL: incremented by n_tokens.
  *   status_dev  device int, may be NULL.
- *   workspace   unused by the current kernels (adadim_workspace_bytes(ADADIM_WS_HESSIAN,..)
- *               is 0); may be NULL.
+ *   workspace   bf16 X: unused, may be NULL.  fp32 X: adadim_workspace_bytes(ADADIM_WS_HESSIAN,
+ *               n_tokens, in, 0, 0) bytes (the chunk's token count in the `out` argument),
+ *               256-byte aligned, for the tensor-core path.
  */
 ADADIM_API int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_tokens, int64_t in, int64_t ldx,
                               float* H, int64_t* n_seen, int* status_dev,

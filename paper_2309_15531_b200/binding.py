@@ -131,12 +131,19 @@ def _ws(nbytes: int, device) -> torch.Tensor:
     return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
 
 
-def hessian_accumulate(X: torch.Tensor, H: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
-    """H += 2 X^T X for X[n_tokens, in] (bf16 or fp32), H[in, in] fp32."""
+def hessian_accumulate(X: torch.Tensor, H: torch.Tensor, status: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None, tensor_cores: bool = True) -> None:
+    """H += 2 X^T X for X[n_tokens, in] (bf16 or fp32), H[in, in] fp32.  fp32 X runs on the tensor cores
+    through a workspace (allocated here if none is given); tensor_cores=False selects the plain kernel."""
     assert X.is_cuda and H.is_cuda and X.stride(1) == 1 and H.is_contiguous()
+    ws_ptr, ws_len = None, 0
+    if X.dtype == torch.float32 and tensor_cores and X.shape[0] > 0:
+        if workspace is None:
+            workspace = _ws(workspace_bytes(WS_HESSIAN, X.shape[0], X.shape[1]), X.device)
+        ws_ptr, ws_len = workspace.data_ptr(), workspace.numel()
     rc = lib().adadim_hessian_accumulate(X.data_ptr(), _DT[X.dtype], X.shape[0], X.shape[1], X.stride(0),
                                          H.data_ptr(), None, status.data_ptr() if status is not None else None,
-                                         None, 0, _stream())
+                                         ws_ptr, ws_len, _stream())
     _check(rc, "adadim_hessian_accumulate")
 
 

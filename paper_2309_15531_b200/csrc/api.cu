@@ -8,6 +8,9 @@ int unpack_launch(const uint32_t* codes, int64_t out, int64_t in, int bits, uint
 int hessian_bf16_launch(const void* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, int* status_dev,
                         cudaStream_t st);
 int hessian_f32_launch(const float* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, cudaStream_t st);
+size_t hessian_f32_tc_workspace_bytes(int64_t n_tokens, int64_t in);
+int hessian_f32_tc_launch(const float* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, int* status_dev,
+                          void* workspace, cudaStream_t st);
 size_t score_workspace_bytes(int64_t out, int64_t in);
 int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw, const float* H, int bits, int group,
                  const adadim_qtensor* q_oc, const adadim_qtensor* q_ic, double* err, int* chosen, int* status_dev,
@@ -108,7 +111,7 @@ size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int g
   (void)bits;
   if (out < 0 || in < 0) return 0;
   switch (kind) {
-    case ADADIM_WS_HESSIAN: return 0;
+    case ADADIM_WS_HESSIAN: return out > 0 ? hessian_f32_tc_workspace_bytes(out, in) : 0;   // out = tokens of an fp32 chunk
     case ADADIM_WS_GPTQ: return gptq_workspace_bytes(2 * out, in);
     case ADADIM_WS_GPTQ_ROWS: return gptq_workspace_bytes(out, in);
     case ADADIM_WS_GEMV: return group > 0 ? gemv_workspace_bytes(out, in, group) : 0;
@@ -121,7 +124,6 @@ size_t adadim_workspace_bytes(int kind, int64_t out, int64_t in, int bits, int g
 int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_tokens, int64_t in, int64_t ldx, float* H,
                               int64_t* n_seen, int* status_dev, void* workspace, size_t workspace_bytes,
                               void* cuda_stream) {
-  (void)workspace; (void)workspace_bytes;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (xdtype != ADADIM_BF16 && xdtype != ADADIM_F32) return ADADIM_ERR_DTYPE;
   if (n_tokens < 0 || in < 0 || ldx < in || in % 8 != 0) return ADADIM_ERR_SHAPE;
@@ -134,8 +136,14 @@ int adadim_hessian_accumulate(const void* X, int xdtype, int64_t n_tokens, int64
   if (X == nullptr) return ADADIM_ERR_NULL;
   const int64_t esz = xdtype == ADADIM_BF16 ? 2 : 4;
   if (!aligned16(X) || (ldx * esz) % 16 != 0) return ADADIM_ERR_ALIGN;
-  if (xdtype == ADADIM_BF16) rc = hessian_bf16_launch(X, n_tokens, in, ldx, H, status_dev, st);
-  else rc = hessian_f32_launch(static_cast<const float*>(X), n_tokens, in, ldx, H, st);
+  if (xdtype == ADADIM_BF16) {
+    rc = hessian_bf16_launch(X, n_tokens, in, ldx, H, status_dev, st);
+  } else if (workspace != nullptr && aligned256(workspace) &&
+             workspace_bytes >= hessian_f32_tc_workspace_bytes(n_tokens, in)) {
+    rc = hessian_f32_tc_launch(static_cast<const float*>(X), n_tokens, in, ldx, H, status_dev, workspace, st);
+  } else {
+    rc = hessian_f32_launch(static_cast<const float*>(X), n_tokens, in, ldx, H, st);
+  }
   if (rc == ADADIM_OK && n_seen != nullptr) *n_seen += n_tokens;
   return rc;
 }

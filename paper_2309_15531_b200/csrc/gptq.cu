@@ -327,7 +327,16 @@ block_kernel(const BlockArgs a) {
   }
   const bool staged = ptx::mbar_wait(&bar[0], 0, &dead_flag, a.status_dev) &
                       ptx::mbar_wait(&bar[1], 0, &dead_flag, a.status_dev);
-  if (!__syncthreads_and(staged)) {
+  bool go = __syncthreads_and(staged) != 0;
+  if (G > kBlk) {
+    // g = 256: the two CTAs of a pair meet at a cluster barrier in every per-IC column, so they go on
+    // or stop together: each tells the other whether its copies arrived
+    if (tid == 0) ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_addr(&xch[3]), ptx::cluster_ctarank() ^ 1u), go ? 1.0f : 0.0f);
+    ptx::cluster_sync();
+    go = go && xch[3] != 0.0f;
+    ptx::cluster_sync();                             // both have read the word before a column's exchange could reuse the array
+  }
+  if (!go) {
     // a copy did not arrive in time (reported as ADADIM_ERR_TIMEOUT): give what is in flight one more
     // bounded wait so that nothing lands in shared memory after the CTA has gone, then stop
     const long long c0 = clock64();

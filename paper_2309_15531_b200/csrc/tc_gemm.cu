@@ -446,6 +446,58 @@ int hessian_bf16_launch(const void* X, int64_t n_tokens, int64_t in, int64_t ldx
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 
+// ---- fp32 activations on the tensor cores ---------------------------------------------------------
+// A binary32 number is the exact sum of three bf16 numbers (8 significant bits each).  With
+// Z = [X_hi | X_mid | X_lo] (the channel axis three times as wide) the bf16 kernel above forms
+// 2 Z^T Z, whose nine in x in blocks are the products 2 X_p^T X_q of the pieces; H gets the six
+// blocks that matter (p + q <= 2; the other three are below 2^-24 of the result), smallest first.
+// Every product of two pieces is exact in the tensor core; what is rounded is the fp32 accumulation,
+// as for bf16 activations.
+namespace {
+__global__ void __launch_bounds__(256)
+split3_kernel(const float* __restrict__ X, int64_t n_tokens, int64_t in, int64_t ldx, __nv_bfloat16* __restrict__ Z) {
+  const int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (e >= n_tokens * in) return;
+  const int64_t t = e / in, i = e % in;
+  const float x = X[t * ldx + i];
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  const float r1 = x - __bfloat162float(h);                  // exact
+  const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+  const float r2 = r1 - __bfloat162float(m);                 // exact
+  __nv_bfloat16* z = Z + t * 3 * in + i;
+  z[0] = h;
+  z[in] = m;
+  z[2 * in] = __float2bfloat16_rn(r2);
+}
+__global__ void __launch_bounds__(256)
+combine3_kernel(const float* __restrict__ Hp, int64_t in, float* __restrict__ H) {
+  const int64_t e = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (e >= in * in) return;
+  const int64_t i = e / in, j = e % in, n3 = 3 * in;
+  auto blk = [&](int p, int q) { return Hp[(p * in + i) * n3 + q * in + j]; };
+  const float small = (blk(0, 2) + blk(2, 0)) + blk(1, 1);
+  const float mid = blk(0, 1) + blk(1, 0);
+  H[e] += (small + mid) + blk(0, 0);
+}
+}  // namespace
+
+size_t hessian_f32_tc_workspace_bytes(int64_t n_tokens, int64_t in) {
+  return round_up(static_cast<size_t>(n_tokens) * 3 * in * 2, 256) + round_up(static_cast<size_t>(9) * in * in * 4, 256);
+}
+
+int hessian_f32_tc_launch(const float* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, int* status_dev,
+                          void* workspace, cudaStream_t st) {
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  __nv_bfloat16* Z = reinterpret_cast<__nv_bfloat16*>(ws);
+  float* Hp = reinterpret_cast<float*>(ws + round_up(static_cast<size_t>(n_tokens) * 3 * in * 2, 256));
+  ADADIM_CUDA_TRY(cudaMemsetAsync(Hp, 0, static_cast<size_t>(9) * in * in * 4, st));
+  split3_kernel<<<static_cast<unsigned>((n_tokens * in + 255) / 256), 256, 0, st>>>(X, n_tokens, in, ldx, Z);
+  const int rc = hessian_bf16_launch(Z, n_tokens, 3 * in, 3 * in, Hp, status_dev, st);
+  if (rc != ADADIM_OK) return rc;
+  combine3_kernel<<<static_cast<unsigned>((in * in + 255) / 256), 256, 0, st>>>(Hp, in, H);
+  return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
+}
+
 int hessian_f32_launch(const float* X, int64_t n_tokens, int64_t in, int64_t ldx, float* H, cudaStream_t st) {
   const int nblk = static_cast<int>((in + 63) / 64);
   hessian_f32_kernel<<<nblk * (nblk + 1) / 2, 256, 0, st>>>(X, n_tokens, in, ldx, H);

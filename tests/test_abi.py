@@ -36,7 +36,8 @@ def test_workspace_sizes_grow_with_the_problem(lib):
     f = lib.adadim_workspace_bytes
     f.restype = ctypes.c_size_t
     f.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int]
-    assert f(0, 4096, 4096, 3, 128) == 0
+    assert f(0, 0, 4096, 3, 128) == 0                              # bf16 activations need no Hessian workspace
+    assert f(0, 256, 512, 0, 0) >= 256 * 3 * 512 * 2 + 9 * 512 * 512 * 4     # an fp32 chunk of 256 tokens: three bf16 pieces + the widened product
     g1, g2 = f(1, 256, 512, 3, 128), f(1, 4096, 4096, 3, 128)
     s1, s2 = f(2, 256, 512, 3, 128), f(2, 4096, 4096, 3, 128)
     assert 0 < g1 < g2 and 0 < s1 < s2

@@ -24,14 +24,32 @@ def _norm_err(H, Href):
     return float(np.max(np.abs(H - Href) / scale))
 
 
-def test_small_fp32_layer():
+@pytest.mark.parametrize("tensor_cores", [True, False])
+def test_small_fp32_layer(tensor_cores):
+    """fp32 activations (configuration 1): on the tensor cores through three exact bf16 pieces, and
+    by the plain multiply-add kernel that serves callers without a workspace."""
     wl = I.workload_small()
     X = I.make_calib(wl["layers"]["linear"][1], "cuda")
     H = torch.zeros(512, 512, device="cuda")
-    B.hessian_accumulate(X, H)
+    st = status_tensor()
+    B.hessian_accumulate(X, H, st, tensor_cores=tensor_cores)
     torch.cuda.synchronize()
+    assert int(st.item()) == 0
     Href = O.hessian(to_np(X))
-    assert _norm_err(to_np(H).astype(np.float64), Href) < 1e-5
+    e = _norm_err(to_np(H).astype(np.float64), Href)
+    print(f"hessian fp32 X, tensor cores {tensor_cores}: normalised max error {e:.3e}")
+    assert e < 1e-5
+
+
+def test_fp32_tensor_core_path_chunks_and_pitch():
+    spec = I.CalibSpec(3000, 384, "f32", "skew", 3, 60.0, 60.0, seed=95)
+    X = I.make_calib(spec, "cuda")
+    Xv = X[:, :320]                                   # pitch 384, width 320
+    H = torch.zeros(320, 320, device="cuda")
+    B.hessian_accumulate(Xv[:1700], H)
+    B.hessian_accumulate(Xv[1700:], H)
+    torch.cuda.synchronize()
+    assert _norm_err(to_np(H).astype(np.float64), O.hessian(to_np(Xv))) < 1e-5
 
 
 @pytest.mark.parametrize("n_tokens,inp", [(1000, 512), (777, 320), (4096, 1024), (130, 64), (64, 8)])
