@@ -264,8 +264,9 @@ GemvLayout gemv_layout(int64_t out, int64_t in, int group) {
   const int64_t groups = group > 0 ? out / group : 0;
   const int nblocks = static_cast<int>(in / kColBlock);
   const int64_t ctas_x = (out + kWarps * kRowsPerWarp - 1) / (kWarps * kRowsPerWarp);
-  // enough CTAs to fill the device (148 SMs) a few times over; the column range is split only when the rows alone do not
-  int splits = ctas_x >= 4 * 148 ? 1 : static_cast<int>((8 * 148 + ctas_x - 1) / (ctas_x > 0 ? ctas_x : 1));
+  // enough warps to cover the memory latency: about 48 per SM (148 SMs), four per CTA; the column range is
+  // split when the rows alone do not provide them
+  int splits = static_cast<int>((148 * 12 + ctas_x - 1) / (ctas_x > 0 ? ctas_x : 1));
   if (splits > nblocks) splits = nblocks;
   if (splits < 1) splits = 1;
   L.blocks_per_split = (nblocks + splits - 1) / splits;
