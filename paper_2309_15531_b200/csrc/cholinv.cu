@@ -27,6 +27,7 @@ constexpr int kNB = 64;     // panel width and small tile edge
 constexpr int kGroup = 4;   // panels per rank-256 update
 
 __host__ __device__ __forceinline__ int64_t mn64(int64_t a, int64_t b) { return a < b ? a : b; }
+__host__ __device__ __forceinline__ int64_t mx64(int64_t a, int64_t b) { return a > b ? a : b; }
 
 // Programmatic dependent launch for the chain of small kernels: a kernel launched with the
 // attribute below may be scheduled while its predecessor in the stream is still finishing; it then
@@ -646,9 +647,9 @@ rank_update_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int
 
 // ---- inverse by recursive doubling -----------------------------------------------------------
 __global__ void __launch_bounds__(256)
-seed_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ dinv) {
-  // diagonal 64-blocks of A <- their inverses
-  const int k = blockIdx.x;
+seed_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ dinv, int k0) {
+  // diagonal 64-blocks k0 + blockIdx.x of A <- their inverses
+  const int k = k0 + blockIdx.x;
   double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
   const double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
   for (int e = threadIdx.x; e < kNB * kNB; e += 256) blk[static_cast<int64_t>(e >> 6) * n + (e & 63)] = dk[e];
@@ -659,10 +660,12 @@ seed_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ dinv) 
 // T is packed pair after pair (every earlier pair has s B-rows), rows local to the B part, pitch s.
 // step 1:  T = C * XA      (T tile (r,c): reduction over XA rows m >= c only, XA is lower)
 // step 2:  C <- -XB * T    (C tile (r,c): reduction over XB columns m <= r only)
+// A launch covers the pairs p0 + blockIdx.{x,y} of one level; the pair's T is slot blockIdx.{x,y}
+// of the level's region (pitch s, s rows per slot).
 __global__ void __launch_bounds__(256)
-merge1_64_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ T) {      // s == 64
+merge1_64_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ T, int p0) {      // s == 64
   TILE_SMEM
-  const int64_t s = kNB, a0 = static_cast<int64_t>(blockIdx.x) * 2 * s, b0 = a0 + s;
+  const int64_t s = kNB, a0 = static_cast<int64_t>(p0 + blockIdx.x) * 2 * s, b0 = a0 + s;
   if (b0 >= n) return;
   double acc[4][2][2] = {};
   tile_product<false>(A + b0 * n + a0, n, A + a0 * n + a0, n, acc, sa, sb);
@@ -672,9 +675,9 @@ merge1_64_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ T
   });
 }
 __global__ void __launch_bounds__(256)
-merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T) {      // s == 64
+merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T, int p0) {      // s == 64
   TILE_SMEM
-  const int64_t s = kNB, a0 = static_cast<int64_t>(blockIdx.x) * 2 * s, b0 = a0 + s;
+  const int64_t s = kNB, a0 = static_cast<int64_t>(p0 + blockIdx.x) * 2 * s, b0 = a0 + s;
   if (b0 >= n) return;
   double acc[4][2][2] = {};
   tile_product<false>(A + b0 * n + b0, n, T + static_cast<int64_t>(blockIdx.x) * s * s, s, acc, sa, sb);
@@ -685,33 +688,33 @@ merge2_64_kernel(double* __restrict__ A, int64_t n, const double* __restrict__ T
 }
 
 __global__ void __launch_bounds__(256, 2)
-merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T) {      // s >= 128
+merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __restrict__ T, int p0) {      // s >= 128
   __shared__ TileSmem64 sm;
-  const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
+  const int64_t a0 = static_cast<int64_t>(p0 + blockIdx.y) * 2 * s, b0 = a0 + s;
   // 64-row block r, 64-column block c; the reduction length s - 64 c falls with c, so tiles are
   // handed out column block by column block: the longest ones start first
   const int rtiles = static_cast<int>(s / kNB);
-  const int r = blockIdx.x % rtiles, c = blockIdx.x / rtiles;
   const int64_t sB = mn64(s, n - b0);
+  const int r = blockIdx.x % rtiles, c = blockIdx.x / rtiles;
   if (static_cast<int64_t>(r) * kNB >= sB) return;
   const int64_t m0 = static_cast<int64_t>(c) * kNB;
   double acc[4][2][2] = {};
   product_tile64<false>(A + (b0 + static_cast<int64_t>(r) * kNB) * n + a0 + m0, n, A + (a0 + m0) * n + a0 + m0, n,
                         static_cast<int>(s - m0), acc, sm);
-  double* t = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kNB * s + m0;
+  double* tp = T + static_cast<int64_t>(blockIdx.y) * s * s + static_cast<int64_t>(r) * kNB * s + m0;
   for_each_pair64(acc, [&](int rr, int c2, const double* v) {
-    *reinterpret_cast<double2*>(t + static_cast<int64_t>(rr) * s + c2) = make_double2(v[0], v[1]);
+    *reinterpret_cast<double2*>(tp + static_cast<int64_t>(rr) * s + c2) = make_double2(v[0], v[1]);
   });
 }
 __global__ void __launch_bounds__(256, 2)
-merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T) {      // s >= 128
+merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T, int p0) {      // s >= 128
   __shared__ TileSmem64 sm;
   const int ctiles = static_cast<int>(s / kNB);
-  const int64_t a0 = static_cast<int64_t>(blockIdx.y) * 2 * s, b0 = a0 + s;
+  const int64_t a0 = static_cast<int64_t>(p0 + blockIdx.y) * 2 * s, b0 = a0 + s;
   // the reduction length 64 (r + 1) grows with the row block: the last row blocks start first
   const int rtiles = static_cast<int>(s / kNB);
-  const int r = rtiles - 1 - static_cast<int>(blockIdx.x) / ctiles, c = blockIdx.x % ctiles;
   const int64_t sB = mn64(s, n - b0);
+  const int r = rtiles - 1 - static_cast<int>(blockIdx.x) / ctiles, c = blockIdx.x % ctiles;
   if (static_cast<int64_t>(r) * kNB >= sB) return;
   const int64_t row0 = b0 + static_cast<int64_t>(r) * kNB;
   const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kNB, sB));
@@ -733,17 +736,94 @@ emit_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ U) {
   U[e] = i <= j ? A[(n - 1 - i) * n + (n - 1 - j)] : 0.0;
 }
 
+// ---- the inverse's schedule ---------------------------------------------------------------------
+// Level l merges with half-size s = 64 << l; pair p of a level covers [p 2s, p 2s + 2s) and exists
+// when its second half starts inside the matrix.  A pair's first step (T = C XA) needs columns
+// [0, p 2s + s) of L final and its first half inverted; its second step needs the whole pair.  The
+// factorization finishes L's columns from the left, so most steps can be issued while it is still
+// running: InverseSchedule::advance(done) issues, level by level, every step that has become
+// possible once columns [0, done) are final.  None of them writes a row or column >= done, and the
+// factorization from there on only reads rows >= done of those columns (its rank updates), so the
+// two never meet; what is left after the last diagonal block is the last pair of every level.
+//
+// A level keeps T for the pairs of ONE first-step launch (`slots` of them, s x s each, s x (n - s)
+// when the matrix is shorter): a new first step is issued only after the second steps of the
+// previous launch, all on one stream.
+constexpr int kMaxLevels = 40;
+struct LevelPlan { int64_t s; int npairs, slots; size_t t_off; };
+struct InversePlan { int nlev; LevelPlan lev[kMaxLevels]; size_t t_doubles; };
+InversePlan inverse_plan(int64_t n) {
+  InversePlan P;
+  P.nlev = 0;
+  size_t off = 0;
+  for (int64_t s = kNB; s < n && P.nlev < kMaxLevels; s *= 2) {
+    LevelPlan& L = P.lev[P.nlev++];
+    L.s = s;
+    L.npairs = static_cast<int>((n - s + 2 * s - 1) / (2 * s));
+    L.slots = static_cast<int>(mx64(1, static_cast<int64_t>(kGroup) * kNB / (2 * s)));
+    L.t_off = off;
+    off += static_cast<size_t>(L.slots > 1 ? L.slots * s * s : s * mn64(s, n - s));
+  }
+  P.t_doubles = off;
+  return P;
+}
+
 struct FactorLayout { size_t a_off, t_off, dinv_off, stats_off, total; };
 FactorLayout factor_layout(int64_t n) {
   FactorLayout L;
   size_t off = 0;
   L.a_off = off;     off += round_up(static_cast<size_t>(n) * n * 8, 256);
-  L.t_off = off;     off += round_up(static_cast<size_t>(n) * (n / 2 + kNB) * 8, 256);
+  L.t_off = off;     off += round_up(inverse_plan(n).t_doubles * 8 + 256, 256);
   L.dinv_off = off;  off += round_up(static_cast<size_t>(n) * kNB * 8, 256);
   L.stats_off = off; off += 256;
   L.total = off;
   return L;
 }
+
+struct InverseSchedule {
+  InversePlan P;
+  double* A;
+  double* T;
+  const double* dinv;
+  int64_t n;
+  int seeded = 0;                                   // diagonal blocks already replaced by their inverses
+  int m1[kMaxLevels] = {}, m2[kMaxLevels] = {}, base[kMaxLevels] = {};   // pairs with step 1 / step 2 issued; first pair of the latest step-1 launch
+  InverseSchedule(double* A_, double* T_, const double* dinv_, int64_t n_) : P(inverse_plan(n_)), A(A_), T(T_), dinv(dinv_), n(n_) {}
+
+  void advance(int64_t done, cudaStream_t st) {
+    const int nbk = static_cast<int>(done / kNB);
+    if (nbk > seeded) {
+      seed_kernel<<<nbk - seeded, 256, 0, st>>>(A, n, dinv, seeded);
+      seeded = nbk;
+    }
+    for (int l = 0; l < P.nlev; ++l) {
+      const LevelPlan& L = P.lev[l];
+      const int64_t s = L.s;
+      double* t = T + L.t_off;
+      const unsigned tiles = static_cast<unsigned>((s / kNB) * (s / kNB));
+      for (;;) {
+        int q2 = m2[l];
+        while (q2 < m1[l] && mn64(static_cast<int64_t>(q2 + 1) * 2 * s, n) <= done) ++q2;
+        if (q2 > m2[l]) {
+          const unsigned cnt = static_cast<unsigned>(q2 - m2[l]);
+          double* ts = t + static_cast<size_t>(m2[l] - base[l]) * s * s;
+          if (s == kNB) merge2_64_kernel<<<cnt, 256, 0, st>>>(A, n, ts, m2[l]);
+          else merge2_kernel<<<dim3(tiles, cnt), 256, 0, st>>>(A, n, s, ts, m2[l]);
+          m2[l] = q2;
+        }
+        if (m2[l] < m1[l]) break;                       // a pair still waits for its second half
+        int q1 = m1[l];
+        while (q1 < L.npairs && q1 - m1[l] < L.slots && static_cast<int64_t>(q1) * 2 * s + s <= done) ++q1;
+        if (q1 == m1[l]) break;
+        const unsigned cnt = static_cast<unsigned>(q1 - m1[l]);
+        if (s == kNB) merge1_64_kernel<<<cnt, 256, 0, st>>>(A, n, t, m1[l]);
+        else merge1_kernel<<<dim3(tiles, cnt), 256, 0, st>>>(A, n, s, t, m1[l]);
+        base[l] = m1[l];
+        m1[l] = q1;
+      }
+    }
+  }
+};
 
 }  // namespace
 
@@ -764,17 +844,21 @@ int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* st
   // rank update of the next group's own columns) runs on a high-priority stream; the rest of each
   // group's rank update runs beside it on a second stream.  Every kernel of the chain fits on an
   // SM next to one CTA of the rank update, so the chain is scheduled as soon as any CTA retires.
+  // The inverse's merges run behind both on a third, lowest-priority stream as soon as the columns
+  // they need are final (InverseSchedule); only the last pair of each level is left when the chain
+  // ends.
   ForkedStreams fs;                                  // joins and releases on every way out of this function
   bool rest_pending = false;
 
   damp_kernel<<<1, 256, 0, st>>>(H, n, percdamp, stats);
   build_kernel<<<eb, 256, 0, st>>>(H, n, stats, perm, A);
   {
-    const int rc = fs.open(st);
+    const int rc = fs.open(st, true);
     if (rc != ADADIM_OK) return rc;
   }
-  cudaStream_t chain = fs.chain, side = fs.side;
+  cudaStream_t chain = fs.chain, side = fs.side, back = fs.back;
   cudaEvent_t ev_panels = fs.ev_a, ev_rest = fs.ev_b;
+  InverseSchedule inv(A, T, dinv, n);
   for (int g0 = 0; g0 < nb; g0 += kGroup) {
     const int g1 = g0 + kGroup < nb ? g0 + kGroup : nb;
     for (int k = g0; k < g1; ++k) {
@@ -785,12 +869,12 @@ int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* st
       if (below > 0 && inner > 0) ADADIM_CUDA_TRY(launch_chained(group_update_kernel, dim3(below, inner), dim3(256), chain, A, n, k));
     }
     const int64_t e = static_cast<int64_t>(g1) * kNB;
+    ADADIM_CUDA_TRY(cudaEventRecord(ev_panels, chain));          // columns [0, e) of L are final
     if (e < n) {
       const int nt = static_cast<int>((n - e + kT - 1) / kT);
       const int64_t j0 = static_cast<int64_t>(g0) * kNB;
       const int kw = (g1 - g0) * kNB;
       const bool has_rest = e + kLook * kTN < n;
-      if (has_rest) ADADIM_CUDA_TRY(cudaEventRecord(ev_panels, chain));
       // the columns updated next were last written by the previous group's side-stream launch
       if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
       ADADIM_CUDA_TRY(launch_chained(rank_update_first_kernel, dim3(kLook, static_cast<unsigned>((n - e) / kNB)), dim3(256), chain, A, n, e, j0, kw));
@@ -802,22 +886,12 @@ int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* st
         rest_pending = true;
       }
     }
+    ADADIM_CUDA_TRY(cudaStreamWaitEvent(back, ev_panels, 0));
+    inv.advance(e < n ? e : n, back);
   }
   {
     const int rc = fs.join();
     if (rc != ADADIM_OK) return rc;
-  }
-  seed_kernel<<<nb, 256, 0, st>>>(A, n, dinv);
-  if (n > kNB) {
-    const unsigned pairs = static_cast<unsigned>((n + 2 * kNB - 1) / (2 * kNB));
-    merge1_64_kernel<<<pairs, 256, 0, st>>>(A, n, T);
-    merge2_64_kernel<<<pairs, 256, 0, st>>>(A, n, T);
-  }
-  for (int64_t s = 2 * kNB; s < n; s *= 2) {
-    const unsigned pairs = static_cast<unsigned>((n + 2 * s - 1) / (2 * s));
-    const unsigned tiles = static_cast<unsigned>((s / kNB) * (s / kNB));
-    merge1_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
-    merge2_kernel<<<dim3(tiles, pairs), 256, 0, st>>>(A, n, s, T);
   }
   emit_kernel<<<eb, 256, 0, st>>>(A, n, U);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;

@@ -37,15 +37,19 @@ int check_score_args(const void* W, int wdtype, int64_t out, int64_t in, int64_t
 // or reuse the workspace in stream order as usual) and releases streams and events; the runtime
 // defers their destruction until the enqueued work has finished.
 struct ForkedStreams {
-  cudaStream_t caller = nullptr, chain = nullptr, side = nullptr;
+  cudaStream_t caller = nullptr, chain = nullptr, side = nullptr, back = nullptr;
   cudaEvent_t ev_a = nullptr, ev_b = nullptr, ev_join = nullptr;
   bool joined = false;
-  int open(cudaStream_t st) {
+  // chain: highest priority; side: one step below it where the device has more than two levels;
+  // back (only with `with_back`): lowest priority, for work that should fill idle SMs only
+  int open(cudaStream_t st, bool with_back = false) {
     caller = st;
     int lo = 0, hi = 0;
     if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaStreamCreateWithPriority(&chain, cudaStreamNonBlocking, hi) != cudaSuccess) return ADADIM_ERR_CUDA;
-    if (cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, lo) != cudaSuccess) return ADADIM_ERR_CUDA;
+    const int mid = with_back && hi + 1 < lo ? lo - 1 : lo;          // numerically lower = more urgent
+    if (cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, mid) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (with_back && cudaStreamCreateWithPriority(&back, cudaStreamNonBlocking, lo) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaEventCreateWithFlags(&ev_a, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaEventCreateWithFlags(&ev_b, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
@@ -53,10 +57,11 @@ struct ForkedStreams {
     if (cudaStreamWaitEvent(chain, ev_join, 0) != cudaSuccess) return ADADIM_ERR_CUDA;
     return ADADIM_OK;
   }
-  // the caller's stream waits for everything enqueued so far on both helper streams
+  // the caller's stream waits for everything enqueued so far on the helper streams
   int join() {
     if (ev_join == nullptr) return ADADIM_ERR_CUDA;
     bool ok = true;
+    if (back != nullptr) ok = cudaEventRecord(ev_join, back) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
     if (side != nullptr) ok = cudaEventRecord(ev_join, side) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
     if (chain != nullptr) ok = cudaEventRecord(ev_join, chain) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
     joined = true;
@@ -69,6 +74,7 @@ struct ForkedStreams {
     if (ev_join != nullptr) cudaEventDestroy(ev_join);
     if (chain != nullptr) cudaStreamDestroy(chain);
     if (side != nullptr) cudaStreamDestroy(side);
+    if (back != nullptr) cudaStreamDestroy(back);
   }
   ForkedStreams() = default;
   ForkedStreams(const ForkedStreams&) = delete;
