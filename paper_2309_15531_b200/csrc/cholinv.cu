@@ -328,14 +328,20 @@ build_kernel(const float* __restrict__ H, int64_t n, const double* __restrict__ 
   A[e] = v;
 }
 
-// One merge level of the in-block inverse (shared memory, 256 threads): for every pair of
-// adjacent SZ x SZ inverted diagonal blocks XA, XB with the block C of the factor between them,
-//   T = C XA,   C <- -XB T.
-// A thread owns SZ/8 elements, a warp one row of T at a time (for SZ = 32), so the first operand
-// is a broadcast and the second is read along a row.  M is zero above the diagonal, which lets
-// both sums run over the whole range with compile-time bounds.
+// ---- diagonal block: Cholesky factor and its inverse, one CTA of 256 threads -------------------
+// Shared memory of the block factorization.  The row pitches are 4 mod 16 doubles, which keeps the
+// fragment loads of the fp64 matrix instruction (8 rows x 4 columns per half-warp) on distinct banks.
+struct PotrfSmem {
+  double M[kNB][kNB + 4];
+  double T[kNB / 2][kNB / 2 + 4];
+  double rdiag[kNB];                       // 1 / L[j][j]
+};
+
+// One merge level of the in-block inverse: for every pair of adjacent SZ x SZ inverted diagonal
+// blocks XA, XB with the block C of the factor between them,  T = C XA,  C <- -XB T.
+// M is zero above the diagonal.  Scalar version (SZ = 8): a thread owns SZ/8 elements.
 template <int SZ>
-__device__ __forceinline__ void merge_level(double (*M)[kNB + 1], double (*T)[kNB / 2 + 1], int tid) {
+__device__ __forceinline__ void merge_level(double (*M)[kNB + 4], double (*T)[kNB / 2 + 4], int tid) {
   constexpr int PER = SZ / 8;
   int gi[PER], jj[PER], a0[PER];
   double acc[PER];
@@ -364,154 +370,130 @@ __device__ __forceinline__ void merge_level(double (*M)[kNB + 1], double (*T)[kN
   for (int u = 0; u < PER; ++u) M[a0[u] + SZ + gi[u] % SZ][a0[u] + jj[u]] = -acc[u];
   __syncthreads();
 }
+// The same level on the fp64 matrix instruction (SZ = 16, 32): 8 x 8 output tiles, warp w takes
+// tiles w, w + 8, ...; the sums skip the k-steps that lie wholly above the diagonal of XA / XB.
+template <int SZ>
+__device__ __forceinline__ void merge_level_mma(double (*M)[kNB + 4], double (*T)[kNB / 2 + 4], int tid) {
+  constexpr int TS = SZ / 8;                       // tiles per side of a pair's block
+  constexpr int NT = (kNB / (2 * SZ)) * TS * TS;   // tiles of the level
+  const int warp = tid >> 5, lane = tid & 31, fr = lane >> 2, fk = lane & 3;
+  for (int t = warp; t < NT; t += 8) {
+    const int p = t / (TS * TS), ti = (t / TS) % TS, tj = t % TS, a0 = p * 2 * SZ;
+    double acc[2] = {0.0, 0.0};
+#pragma unroll
+    for (int k0 = 0; k0 < SZ; k0 += 4)
+      if (k0 + 4 > tj * 8) mma_f64(acc, M[a0 + SZ + ti * 8 + fr][a0 + k0 + fk], M[a0 + k0 + fk][a0 + tj * 8 + fr]);
+    T[p * SZ + ti * 8 + fr][tj * 8 + 2 * fk] = acc[0];
+    T[p * SZ + ti * 8 + fr][tj * 8 + 2 * fk + 1] = acc[1];
+  }
+  __syncthreads();
+  for (int t = warp; t < NT; t += 8) {
+    const int p = t / (TS * TS), ti = (t / TS) % TS, tj = t % TS, a0 = p * 2 * SZ;
+    double acc[2] = {0.0, 0.0};
+#pragma unroll
+    for (int k0 = 0; k0 < SZ; k0 += 4)
+      if (k0 < (ti + 1) * 8) mma_f64(acc, M[a0 + SZ + ti * 8 + fr][a0 + SZ + k0 + fk], T[p * SZ + k0 + fk][tj * 8 + fr]);
+    M[a0 + SZ + ti * 8 + fr][a0 + tj * 8 + 2 * fk] = -acc[0];
+    M[a0 + SZ + ti * 8 + fr][a0 + tj * 8 + 2 * fk + 1] = -acc[1];
+  }
+  __syncthreads();
+}
 
-// ---- factorization -------------------------------------------------------------------------
-// Diagonal block k: in-place Cholesky of the 64 x 64 block and its triangular inverse -> dinv[k].
+// In-place Cholesky of the 64 x 64 block held in s.M (its lower triangle; what is above the
+// diagonal is ignored) and the triangular inverse of the factor.  On return the factor is in
+// blk (row pitch n, zeros above the diagonal) and the inverse in dk (64 x 64, pitch 64).  Every
+// thread of the CTA calls it, after a barrier that follows the writes to s.M.
 // The block is worked in eight sub-panels of eight columns, right-looking inside shared memory:
-//   (a) every thread factors the 8 x 8 diagonal piece redundantly in registers (the sequential
-//       chain of eight reciprocal square roots then needs no exchange between threads), and the
-//       thread that owns a row below solves its 8 entries by substitution;
-//   (b) rank-8 update of the rows and columns after the sub-panel.
+//   (a) warps 0 and 1: every thread factors the 8 x 8 diagonal piece redundantly in registers (the
+//       sequential chain of eight reciprocal square roots then needs no exchange between threads)
+//       and solves the row it owns below the piece by substitution, step by step with the chain;
+//   (b) rank-8 update of what follows on the fp64 matrix instruction in 8 x 8 tiles: the next
+//       eight columns first (one tile per warp), then, while (a) already runs on them, the rest
+//       on the other six warps.
 // The inverse is built in place by recursive doubling: 8 x 8 diagonal pieces by substitution
 // (one warp each, one column per lane), then three merge levels
 //   inv([[A,0],[C,B]]) = [[A^-1,0],[-B^-1 C A^-1,B^-1]].
-__global__ void __launch_bounds__(256, 2)
-potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv, int* status_dev) {
+__device__ __forceinline__ void potrf_block(PotrfSmem& s, double* __restrict__ blk, int64_t n,
+                                            double* __restrict__ dk, int* status_dev) {
   constexpr int kSub = 8;
-  __shared__ double M[kNB][kNB + 1];
-  __shared__ double T[kNB / 2][kNB / 2 + 1];
-  __shared__ double rdiag[kNB];          // 1 / L[j][j]
+  double (*M)[kNB + 4] = s.M;
+  double (*T)[kNB / 2 + 4] = s.T;
+  double* rdiag = s.rdiag;
   const int tid = threadIdx.x;
-  double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
-  dep_release();
-  dep_wait();
-  {
-    double v[kNB * kNB / 256];                         // all loads in flight before the first store
-#pragma unroll
-    for (int u = 0; u < kNB * kNB / 256; ++u) {
-      const int e = tid + 256 * u;
-      v[u] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
-    }
-#pragma unroll
-    for (int u = 0; u < kNB * kNB / 256; ++u) {
-      const int e = tid + 256 * u;
-      M[e >> 6][e & 63] = v[u];
-    }
-  }
-  __syncthreads();
-
-  // Sub-panel j's factor-and-solve (a) depends only on the next eight columns of the block.  After
-  // each sub-panel the two warps that run (a) therefore update just those columns (b1) and go
-  // straight on to the next (a), while the other six warps update the rest of the block (b2).
-  double d[kSub][kSub], rinv[kSub], x[kSub];
+  double d[kSub][kSub], x[kSub];
   bool bad = false;
-  // (a): the 8 x 8 diagonal piece at j0, factored in registers by every thread of warps 0 and 1,
-  // and the thread's row below it solved by substitution (finished entries pushed forward)
   auto factor_and_solve = [&](int j0) {
     const int row = j0 + kSub + tid;
 #pragma unroll
     for (int r = 0; r < kSub; ++r)
 #pragma unroll
       for (int c = 0; c <= r; ++c) d[r][c] = M[j0 + r][j0 + c];
-    if (row < kNB) {
 #pragma unroll
-      for (int c = 0; c < kSub; ++c) x[c] = M[row][j0 + c];
-    }
+    for (int c = 0; c < kSub; ++c) x[c] = row < kNB ? M[row][j0 + c] : 0.0;
 #pragma unroll
     for (int c = 0; c < kSub; ++c) {
       double piv = d[c][c];
       if (!(piv > 0.0)) { bad = true; piv = 1.0; }
       const double r = rsqrt(piv);
-      rinv[c] = r;
+      if (tid == 63) rdiag[j0 + c] = r;
       d[c][c] = piv * r;
+      x[c] *= r;
 #pragma unroll
       for (int r2 = c + 1; r2 < kSub; ++r2) d[r2][c] *= r;
 #pragma unroll
-      for (int c2 = c + 1; c2 < kSub; ++c2)
+      for (int c2 = c + 1; c2 < kSub; ++c2) {
 #pragma unroll
         for (int r2 = c2; r2 < kSub; ++r2) d[r2][c2] = fma(-d[r2][c], d[c2][c], d[r2][c2]);
-    }
-    if (row < kNB) {
-#pragma unroll
-      for (int c = 0; c < kSub; ++c) {
-        x[c] *= rinv[c];
-#pragma unroll
-        for (int c2 = c + 1; c2 < kSub; ++c2) x[c2] = fma(-x[c], d[c2][c], x[c2]);
+        x[c2] = fma(-x[c], d[c2][c], x[c2]);
       }
     }
   };
-  // results of (a) at j0 into M: each row owner its row, one thread the diagonal piece
-  auto write_back = [&](int j0) {
+  auto store_results = [&](int j0) {                   // of factor_and_solve(j0), by the threads that ran it
     const int row = j0 + kSub + tid;
     if (row < kNB) {
 #pragma unroll
       for (int c = 0; c < kSub; ++c) M[row][j0 + c] = x[c];
     } else if (tid == 63) {                            // never owns a row: j0 + 8 + 63 > 63
 #pragma unroll
-      for (int r = 0; r < kSub; ++r) {
+      for (int r = 0; r < kSub; ++r)
 #pragma unroll
         for (int c = 0; c <= r; ++c) M[j0 + r][j0 + c] = d[r][c];
-        rdiag[j0 + r] = rinv[r];
-      }
       if (bad) report(status_dev, ADADIM_ERR_NOT_PD);
     }
   };
+  // M[r0 .. r0+8)[c0 .. c0+8) -= M[r0 ..][j0 .. j0+8) M[c0 ..][j0 .. j0+8)^T, one warp
+  auto update_tile = [&](int j0, int r0, int c0) {
+    const int lane = tid & 31, fr = lane >> 2, fk = lane & 3;
+    const double a0 = M[r0 + fr][j0 + fk], a1 = M[r0 + fr][j0 + 4 + fk];
+    const double b0 = M[c0 + fr][j0 + fk], b1 = M[c0 + fr][j0 + 4 + fk];
+    double2* o = reinterpret_cast<double2*>(&M[r0 + fr][c0 + 2 * fk]);
+    const double2 ov = *o;
+    double p[2] = {0.0, 0.0}, q[2] = {0.0, 0.0};
+    mma_f64(p, a0, b0);
+    mma_f64(q, a1, b1);
+    *o = make_double2(ov.x - (p[0] + q[0]), ov.y - (p[1] + q[1]));
+  };
 
-  if (tid < 64) factor_and_solve(0);
-  __syncthreads();                                     // every thread has read the old piece
-  if (tid < 64) write_back(0);
+  if (tid < 64) { factor_and_solve(0); store_results(0); }
   __syncthreads();
 #pragma unroll 1
   for (int j0 = 0; j0 + kSub < kNB; j0 += kSub) {
-    const int lim = j0 + kSub;
+    const int lim = j0 + kSub, warp = tid >> 5;
+    const int m = (kNB - lim) / kSub;                  // 8 x 8 tiles per side of what is left
+    if (warp < m) update_tile(j0, lim + warp * kSub, lim);
+    __syncthreads();
     if (tid < 64) {
-      // (b1) M[r][lim + c] -= sum_m M[r][j0+m] M[lim+c][j0+m] for the next eight columns, one row per thread
-      const int r = lim + tid;
-      if (r < kNB) {
-        double am[kSub], acc[kSub];
-#pragma unroll
-        for (int m = 0; m < kSub; ++m) am[m] = M[r][j0 + m];
-#pragma unroll
-        for (int c = 0; c < kSub; ++c) {
-          acc[c] = 0.0;
-#pragma unroll
-          for (int m = 0; m < kSub; ++m) acc[c] = fma(am[m], M[lim + c][j0 + m], acc[c]);
-        }
-#pragma unroll
-        for (int c = 0; c < kSub; ++c)
-          if (lim + c <= r) M[r][lim + c] -= acc[c];
-      }
-      asm volatile("bar.sync 1, 64;" ::: "memory");    // warps 0 and 1 only
       factor_and_solve(lim);
+      store_results(lim);                              // columns lim .. lim+7: no tile of the branch below touches them
     } else {
-      // (b2) the same update for the columns after those, lim + 8 <= c <= r, on the other 192 threads:
-      // thread (ty, tx) owns rows ty + 12 i and columns tx + 16 j
-      const int t2 = tid - 64, tx = t2 & 15, ty = t2 >> 4;
-      if (lim + kSub < kNB) {
-        double acc[6][4] = {};
-#pragma unroll
-        for (int m = 0; m < kSub; ++m) {
-          double av[6], bv[4];
-#pragma unroll
-          for (int i = 0; i < 6; ++i) av[i] = ty + 12 * i < kNB ? M[ty + 12 * i][j0 + m] : 0.0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) bv[j] = M[tx + 16 * j][j0 + m];
-#pragma unroll
-          for (int i = 0; i < 6; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
-        }
-#pragma unroll
-        for (int i = 0; i < 6; ++i)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int r = ty + 12 * i, c = tx + 16 * j;
-            if (r < kNB && c >= lim + kSub && c <= r) M[r][c] -= acc[i][j];
-          }
+      // tile t = ti (ti - 1) / 2 + (tj - 1), 1 <= tj <= ti < m, on warps 2..7
+      for (int t = warp - 2; t < m * (m - 1) / 2; t += 6) {
+        int ti = 1;
+        while (t >= ti * (ti + 1) / 2) ++ti;
+        const int tj = t - ti * (ti - 1) / 2 + 1;
+        update_tile(j0, lim + ti * kSub, lim + tj * kSub);
       }
     }
-    __syncthreads();                                   // (b2) done; every thread of (a) has read its inputs
-    if (tid < 64) write_back(lim);
     __syncthreads();
   }
 
@@ -531,12 +513,14 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
     const int o = wv * kSub;
     double xx[kSub];
     if (c < kSub) {
+      // column c by forward substitution, finished entries pushed forward
+#pragma unroll
+      for (int r = 0; r < kSub; ++r) xx[r] = r == c ? 1.0 : 0.0;
 #pragma unroll
       for (int r = 0; r < kSub; ++r) {
-        double sacc = 0.0;
+        xx[r] *= rdiag[o + r];
 #pragma unroll
-        for (int m = 0; m < r; ++m) sacc = fma(M[o + r][o + m], xx[m], sacc);   // xx[m] == 0 for m < c
-        xx[r] = r < c ? 0.0 : ((r == c ? 1.0 : 0.0) - sacc) * rdiag[o + r];
+        for (int r2 = r + 1; r2 < kSub; ++r2) xx[r2] = fma(-M[o + r2][o + r], xx[r], xx[r2]);
       }
     }
     __syncwarp();
@@ -547,13 +531,38 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
   }
   __syncthreads();
   merge_level<8>(M, T, tid);
-  merge_level<16>(M, T, tid);
-  merge_level<32>(M, T, tid);
-  double* dk = dinv + static_cast<int64_t>(k) * kNB * kNB;
+  merge_level_mma<16>(M, T, tid);
+  merge_level_mma<32>(M, T, tid);
   for (int e = tid; e < kNB * kNB; e += 256) {
     const int r = e >> 6, c = e & 63;
     dk[e] = r >= c ? M[r][c] : 0.0;
   }
+}
+
+// Diagonal block k as a launch of its own (block 0; every later one is factored by the CTA that
+// finishes its last update, see group_update_kernel and rank_update_first_kernel).
+__global__ void __launch_bounds__(256, 2)
+potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv, int* status_dev) {
+  __shared__ PotrfSmem s;
+  const int tid = threadIdx.x;
+  double* blk = A + (static_cast<int64_t>(k) * kNB) * n + static_cast<int64_t>(k) * kNB;
+  dep_release();
+  dep_wait();
+  {
+    double v[kNB * kNB / 256];                         // all loads in flight before the first store
+#pragma unroll
+    for (int u = 0; u < kNB * kNB / 256; ++u) {
+      const int e = tid + 256 * u;
+      v[u] = blk[static_cast<int64_t>(e >> 6) * n + (e & 63)];
+    }
+#pragma unroll
+    for (int u = 0; u < kNB * kNB / 256; ++u) {
+      const int e = tid + 256 * u;
+      s.M[e >> 6][e & 63] = v[u];
+    }
+  }
+  __syncthreads();
+  potrf_block(s, blk, n, dinv + static_cast<int64_t>(k) * kNB * kNB, status_dev);
 }
 
 // Panel below diagonal block k:  A[i][k] <- A[i][k] * inv(L_kk)^T   (one 64-row tile per CTA)
