@@ -566,8 +566,12 @@ potrf_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv
 }
 
 // Panel below diagonal block k:  A[i][k] <- A[i][k] * inv(L_kk)^T   (one 64-row tile per CTA)
+// The kernels of the chain start before their predecessor has finished (programmatic dependent
+// launch) and wait for it inside, so what the predecessor writes is not read-only for the kernel's
+// lifetime: `dinv` must not be `const __restrict__`, which would let its loads be treated as
+// invariant and moved above the wait.
 __global__ void __launch_bounds__(256)
-panel_kernel(double* __restrict__ A, int64_t n, int k, const double* __restrict__ dinv) {
+panel_kernel(double* __restrict__ A, int64_t n, int k, const double* dinv) {
   TILE_SMEM
   const int64_t row0 = (static_cast<int64_t>(k) + 1 + blockIdx.x) * kNB;
   double* tile = A + row0 * n + static_cast<int64_t>(k) * kNB;
@@ -583,9 +587,15 @@ panel_kernel(double* __restrict__ A, int64_t n, int k, const double* __restrict_
 // Update inside the current group of panels after panel k:  A[i][j] -= L[i][k] L[j][k]^T for the
 // column tiles j of the group that follow k and all row tiles i >= j.  blockIdx.x = i - (k+1),
 // blockIdx.y = j - (k+1).
-__global__ void __launch_bounds__(256)
-group_update_kernel(double* __restrict__ A, int64_t n, int k) {
-  TILE_SMEM
+// The CTA of tile (k+1, k+1) then holds the next diagonal block in its final state: it does not
+// store it but factors it on the spot (potrf_block), so that the chain goes on without a launch
+// and a round trip through memory in between, while the other CTAs finish their tiles.
+__global__ void __launch_bounds__(256, 2)
+group_update_kernel(double* __restrict__ A, int64_t n, int k, double* __restrict__ dinv, int* status_dev) {
+  __shared__ __align__(16) unsigned char raw[sizeof(PotrfSmem)];
+  static_assert(sizeof(PotrfSmem) >= 2 * kHalfK * (kNB + 4) * sizeof(double), "tile staging fits");
+  double (*sa)[kNB + 4] = reinterpret_cast<double (*)[kNB + 4]>(raw);
+  double (*sb)[kNB + 4] = sa + kHalfK;
   dep_release();
   dep_wait();
   if (blockIdx.y > blockIdx.x) return;
@@ -594,6 +604,17 @@ group_update_kernel(double* __restrict__ A, int64_t n, int k) {
   double acc[4][2][2] = {};
   tile_product<true>(A + ri * n + ck, n, A + rj * n + ck, n, acc, sa, sb);
   double* c0 = A + ri * n + rj;
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
+    PotrfSmem& s = *reinterpret_cast<PotrfSmem*>(raw);
+    __syncthreads();                                   // the staged operands have been read by every warp
+    for_each_pair64(acc, [&](int r, int c, const double* v) {
+      const double2 u = *reinterpret_cast<const double2*>(c0 + static_cast<int64_t>(r) * n + c);
+      *reinterpret_cast<double2*>(&s.M[r][c]) = make_double2(u.x - v[0], u.y - v[1]);
+    });
+    __syncthreads();
+    potrf_block(s, c0, n, dinv + (static_cast<int64_t>(k) + 1) * kNB * kNB, status_dev);
+    return;
+  }
   for_each_pair64(acc, [&](int r, int c, const double* v) {
     double2* p = reinterpret_cast<double2*>(c0 + static_cast<int64_t>(r) * n + c);
     double2 u = *p;
@@ -606,14 +627,18 @@ group_update_kernel(double* __restrict__ A, int64_t n, int k) {
 //   A[i][j] -= L[i][j0 .. j0+kw) L[j][j0 .. j0+kw)^T   on and below the diagonal.
 // The update is issued in two parts so that the next group's factorization can start early:
 //  * the next group's own columns [e, e + 256): rank_update_first_kernel, 64 x 64 tiles, one wave
-//    of short CTAs on the high-priority chain;
+//    of short CTAs on the high-priority chain; the CTA of the first diagonal tile goes straight on
+//    to factor it (as in group_update_kernel);
 //  * the rest: rank_update_kernel, 128 x 64 tiles over the whole triangle, skipping those columns.
 // In the second kernel row block ti meets column blocks 0 .. 2*ti+1; the tile right of the diagonal
 // 64-block (column block 2*ti+1) only stores its lower 64 rows: the block above them must stay zero.
 constexpr int kLook = kGroup * kNB / kTN;
 __global__ void __launch_bounds__(256, 2)
-rank_update_first_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw) {
-  __shared__ TileSmem64 sm;
+rank_update_first_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j0, int kw,
+                         double* __restrict__ dinv, int* status_dev) {
+  __shared__ __align__(16) unsigned char raw[sizeof(PotrfSmem)];
+  static_assert(sizeof(PotrfSmem) >= sizeof(TileSmem64), "tile staging fits");
+  TileSmem64& sm = *reinterpret_cast<TileSmem64*>(raw);
   const int ti = blockIdx.y, cj = blockIdx.x;               // 64-row block, 64-column block of the region
   dep_release();
   dep_wait();
@@ -622,6 +647,19 @@ rank_update_first_kernel(double* __restrict__ A, int64_t n, int64_t e, int64_t j
   if (rj >= n) return;
   double acc[4][2][2] = {};
   product_tile64<true>(A + ri * n + j0, n, A + rj * n + j0, n, kw, acc, sm);
+  if (ti == 0 && cj == 0) {
+    // the next group's first diagonal block is final with this update: factor it here
+    PotrfSmem& s = *reinterpret_cast<PotrfSmem*>(raw);
+    double* blk = A + ri * n + rj;
+    __syncthreads();                                   // the staged slabs have been read by every warp
+    for_each_pair64(acc, [&](int r, int c2, const double* v) {
+      const double2 u = *reinterpret_cast<const double2*>(blk + static_cast<int64_t>(r) * n + c2);
+      *reinterpret_cast<double2*>(&s.M[r][c2]) = make_double2(u.x - v[0], u.y - v[1]);
+    });
+    __syncthreads();
+    potrf_block(s, blk, n, dinv + (e / kNB) * kNB * kNB, status_dev);
+    return;
+  }
   for_each_pair64(acc, [&](int r, int c2, const double* v) {
     double2* p = reinterpret_cast<double2*>(A + (ri + r) * n + rj + c2);
     double2 u = *p;
@@ -799,15 +837,27 @@ struct InverseSchedule {
   int m1[kMaxLevels] = {}, m2[kMaxLevels] = {}, base[kMaxLevels] = {};   // pairs with step 1 / step 2 issued; first pair of the latest step-1 launch
   InverseSchedule(double* A_, double* T_, const double* dinv_, int64_t n_) : P(inverse_plan(n_)), A(A_), T(T_), dinv(dinv_), n(n_) {}
 
-  void advance(int64_t done, cudaStream_t st) {
+  // The levels up to half-size kSmallLevel are short launches of a few CTAs, bound by their
+  // latency; the levels above them are long and bound by throughput.  They go to two streams
+  // (`st`, `st_big`) so that the second kind runs beside the first; `ev` carries the dependency
+  // of a level on the ones below it across the two.
+  static constexpr int64_t kSmallLevel = 256;
+  int advance(int64_t done, cudaStream_t st_small, cudaStream_t st_big, cudaEvent_t ev) {
     const int nbk = static_cast<int>(done / kNB);
     if (nbk > seeded) {
-      seed_kernel<<<nbk - seeded, 256, 0, st>>>(A, n, dinv, seeded);
+      seed_kernel<<<nbk - seeded, 256, 0, st_small>>>(A, n, dinv, seeded);
       seeded = nbk;
     }
+    bool crossed = false;
     for (int l = 0; l < P.nlev; ++l) {
       const LevelPlan& L = P.lev[l];
       const int64_t s = L.s;
+      cudaStream_t st = s <= kSmallLevel ? st_small : st_big;
+      if (s > kSmallLevel && !crossed) {
+        crossed = true;
+        ADADIM_CUDA_TRY(cudaEventRecord(ev, st_small));
+        ADADIM_CUDA_TRY(cudaStreamWaitEvent(st_big, ev, 0));
+      }
       double* t = T + L.t_off;
       const unsigned tiles = static_cast<unsigned>((s / kNB) * (s / kNB));
       for (;;) {
@@ -831,6 +881,7 @@ struct InverseSchedule {
         m1[l] = q1;
       }
     }
+    return ADADIM_OK;
   }
 };
 
@@ -871,11 +922,12 @@ int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* st
   for (int g0 = 0; g0 < nb; g0 += kGroup) {
     const int g1 = g0 + kGroup < nb ? g0 + kGroup : nb;
     for (int k = g0; k < g1; ++k) {
-      ADADIM_CUDA_TRY(launch_chained(potrf_kernel, dim3(1), dim3(256), chain, A, n, k, dinv, status_dev));
+      // diagonal block k > 0 was factored by the launch that completed it
+      if (k == 0) ADADIM_CUDA_TRY(launch_chained(potrf_kernel, dim3(1), dim3(256), chain, A, n, k, dinv, status_dev));
       const int below = nb - k - 1;
       if (below > 0) ADADIM_CUDA_TRY(launch_chained(panel_kernel, dim3(below), dim3(256), chain, A, n, k, static_cast<const double*>(dinv)));
       const int inner = g1 - k - 1;
-      if (below > 0 && inner > 0) ADADIM_CUDA_TRY(launch_chained(group_update_kernel, dim3(below, inner), dim3(256), chain, A, n, k));
+      if (below > 0 && inner > 0) ADADIM_CUDA_TRY(launch_chained(group_update_kernel, dim3(below, inner), dim3(256), chain, A, n, k, dinv, status_dev));
     }
     const int64_t e = static_cast<int64_t>(g1) * kNB;
     ADADIM_CUDA_TRY(cudaEventRecord(ev_panels, chain));          // columns [0, e) of L are final
@@ -886,7 +938,7 @@ int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* st
       const bool has_rest = e + kLook * kTN < n;
       // the columns updated next were last written by the previous group's side-stream launch
       if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
-      ADADIM_CUDA_TRY(launch_chained(rank_update_first_kernel, dim3(kLook, static_cast<unsigned>((n - e) / kNB)), dim3(256), chain, A, n, e, j0, kw));
+      ADADIM_CUDA_TRY(launch_chained(rank_update_first_kernel, dim3(kLook, static_cast<unsigned>((n - e) / kNB)), dim3(256), chain, A, n, e, j0, kw, dinv, status_dev));
       rest_pending = false;
       if (has_rest) {
         ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_panels, 0));
@@ -896,7 +948,10 @@ int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* st
       }
     }
     ADADIM_CUDA_TRY(cudaStreamWaitEvent(back, ev_panels, 0));
-    inv.advance(e < n ? e : n, back);
+    {
+      const int rc = inv.advance(e < n ? e : n, back, fs.back2, fs.ev_c);
+      if (rc != ADADIM_OK) return rc;
+    }
   }
   {
     const int rc = fs.join();

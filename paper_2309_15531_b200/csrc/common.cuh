@@ -37,11 +37,11 @@ int check_score_args(const void* W, int wdtype, int64_t out, int64_t in, int64_t
 // or reuse the workspace in stream order as usual) and releases streams and events; the runtime
 // defers their destruction until the enqueued work has finished.
 struct ForkedStreams {
-  cudaStream_t caller = nullptr, chain = nullptr, side = nullptr, back = nullptr;
-  cudaEvent_t ev_a = nullptr, ev_b = nullptr, ev_join = nullptr;
+  cudaStream_t caller = nullptr, chain = nullptr, side = nullptr, back = nullptr, back2 = nullptr;
+  cudaEvent_t ev_a = nullptr, ev_b = nullptr, ev_c = nullptr, ev_join = nullptr;
   bool joined = false;
   // chain: highest priority; side: one step below it where the device has more than two levels;
-  // back (only with `with_back`): lowest priority, for work that should fill idle SMs only
+  // back, back2 (only with `with_back`): lowest priority, for work that should fill idle SMs only
   int open(cudaStream_t st, bool with_back = false) {
     caller = st;
     int lo = 0, hi = 0;
@@ -50,6 +50,8 @@ struct ForkedStreams {
     const int mid = with_back && hi + 1 < lo ? lo - 1 : lo;          // numerically lower = more urgent
     if (cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, mid) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (with_back && cudaStreamCreateWithPriority(&back, cudaStreamNonBlocking, lo) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (with_back && cudaStreamCreateWithPriority(&back2, cudaStreamNonBlocking, lo) != cudaSuccess) return ADADIM_ERR_CUDA;
+    if (with_back && cudaEventCreateWithFlags(&ev_c, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaEventCreateWithFlags(&ev_a, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaEventCreateWithFlags(&ev_b, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
     if (cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess) return ADADIM_ERR_CUDA;
@@ -61,6 +63,7 @@ struct ForkedStreams {
   int join() {
     if (ev_join == nullptr) return ADADIM_ERR_CUDA;
     bool ok = true;
+    if (back2 != nullptr) ok = cudaEventRecord(ev_join, back2) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
     if (back != nullptr) ok = cudaEventRecord(ev_join, back) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
     if (side != nullptr) ok = cudaEventRecord(ev_join, side) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
     if (chain != nullptr) ok = cudaEventRecord(ev_join, chain) == cudaSuccess && cudaStreamWaitEvent(caller, ev_join, 0) == cudaSuccess && ok;
@@ -71,10 +74,12 @@ struct ForkedStreams {
     if (!joined && ev_join != nullptr) join();
     if (ev_a != nullptr) cudaEventDestroy(ev_a);
     if (ev_b != nullptr) cudaEventDestroy(ev_b);
+    if (ev_c != nullptr) cudaEventDestroy(ev_c);
     if (ev_join != nullptr) cudaEventDestroy(ev_join);
     if (chain != nullptr) cudaStreamDestroy(chain);
     if (side != nullptr) cudaStreamDestroy(side);
     if (back != nullptr) cudaStreamDestroy(back);
+    if (back2 != nullptr) cudaStreamDestroy(back2);
   }
   ForkedStreams() = default;
   ForkedStreams(const ForkedStreams&) = delete;
