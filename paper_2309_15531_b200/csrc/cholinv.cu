@@ -753,16 +753,17 @@ merge1_kernel(const double* __restrict__ A, int64_t n, int64_t s, double* __rest
     *reinterpret_cast<double2*>(tp + static_cast<int64_t>(rr) * s + c2) = make_double2(v[0], v[1]);
   });
 }
+// Rows [64 r_lo, 64 r_hi) of the pair's lower-left block only: row block r of the result needs rows
+// <= r of XB, which are final as soon as the factorization has passed them.
 __global__ void __launch_bounds__(256, 2)
-merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T, int p0) {      // s >= 128
+merge2_kernel(double* __restrict__ A, int64_t n, int64_t s, const double* __restrict__ T, int p0, int r_lo, int r_hi) {      // s >= 128
   __shared__ TileSmem64 sm;
   const int ctiles = static_cast<int>(s / kNB);
   const int64_t a0 = static_cast<int64_t>(p0 + blockIdx.y) * 2 * s, b0 = a0 + s;
   // the reduction length 64 (r + 1) grows with the row block: the last row blocks start first
-  const int rtiles = static_cast<int>(s / kNB);
+  const int r = r_hi - 1 - static_cast<int>(blockIdx.x) / ctiles, c = blockIdx.x % ctiles;
   const int64_t sB = mn64(s, n - b0);
-  const int r = rtiles - 1 - static_cast<int>(blockIdx.x) / ctiles, c = blockIdx.x % ctiles;
-  if (static_cast<int64_t>(r) * kNB >= sB) return;
+  if (r < r_lo || static_cast<int64_t>(r) * kNB >= sB) return;
   const int64_t row0 = b0 + static_cast<int64_t>(r) * kNB;
   const int K = static_cast<int>(mn64(static_cast<int64_t>(r + 1) * kNB, sB));
   double acc[4][2][2] = {};
@@ -792,6 +793,10 @@ emit_kernel(const double* __restrict__ A, int64_t n, double* __restrict__ U) {
 // possible once columns [0, done) are final.  None of them writes a row or column >= done, and the
 // factorization from there on only reads rows >= done of those columns (its rank updates), so the
 // two never meet; what is left after the last diagonal block is the last pair of every level.
+//
+// Above half-size 256 a pair's second step is itself issued in slices of rows: row block r of
+// -XB T needs rows <= r of XB only, and those are final once the factorization has passed them (the
+// lower levels, issued first, have completed them up to the same point).
 //
 // A level keeps T for the pairs of ONE first-step launch (`slots` of them, s x s each, s x (n - s)
 // when the matrix is shorter): a new first step is issued only after the second steps of the
@@ -835,6 +840,7 @@ struct InverseSchedule {
   int64_t n;
   int seeded = 0;                                   // diagonal blocks already replaced by their inverses
   int m1[kMaxLevels] = {}, m2[kMaxLevels] = {}, base[kMaxLevels] = {};   // pairs with step 1 / step 2 issued; first pair of the latest step-1 launch
+  int rows2[kMaxLevels] = {};                       // 64-row blocks of pair m2's second step already issued (levels above kSmallLevel)
   InverseSchedule(double* A_, double* T_, const double* dinv_, int64_t n_) : P(inverse_plan(n_)), A(A_), T(T_), dinv(dinv_), n(n_) {}
 
   // The levels up to half-size kSmallLevel are short launches of a few CTAs, bound by their
@@ -861,14 +867,31 @@ struct InverseSchedule {
       double* t = T + L.t_off;
       const unsigned tiles = static_cast<unsigned>((s / kNB) * (s / kNB));
       for (;;) {
-        int q2 = m2[l];
-        while (q2 < m1[l] && mn64(static_cast<int64_t>(q2 + 1) * 2 * s, n) <= done) ++q2;
-        if (q2 > m2[l]) {
-          const unsigned cnt = static_cast<unsigned>(q2 - m2[l]);
-          double* ts = t + static_cast<size_t>(m2[l] - base[l]) * s * s;
-          if (s == kNB) merge2_64_kernel<<<cnt, 256, 0, st>>>(A, n, ts, m2[l]);
-          else merge2_kernel<<<dim3(tiles, cnt), 256, 0, st>>>(A, n, s, ts, m2[l]);
-          m2[l] = q2;
+        if (s > kSmallLevel) {
+          // one pair at a time, its second step in row slices as the factorization passes them
+          if (m2[l] < m1[l]) {
+            const int q = m2[l];
+            const int64_t b0 = static_cast<int64_t>(q) * 2 * s + s, sB = mn64(s, n - b0);
+            int avail = static_cast<int>((mn64(done, b0 + sB) - b0) / kNB);
+            const int half = static_cast<int>(s / (2 * kNB));                  // slices of half the block: short slices fill the machine badly
+            if (static_cast<int64_t>(avail) * kNB < sB) avail = avail / half * half;
+            if (avail > rows2[l]) {
+              const unsigned gx = static_cast<unsigned>((avail - rows2[l]) * (s / kNB));
+              merge2_kernel<<<dim3(gx, 1), 256, 0, st>>>(A, n, s, t, q, rows2[l], avail);
+              rows2[l] = avail;
+            }
+            if (static_cast<int64_t>(rows2[l]) * kNB >= sB) { ++m2[l]; rows2[l] = 0; }
+          }
+        } else {
+          int q2 = m2[l];
+          while (q2 < m1[l] && mn64(static_cast<int64_t>(q2 + 1) * 2 * s, n) <= done) ++q2;
+          if (q2 > m2[l]) {
+            const unsigned cnt = static_cast<unsigned>(q2 - m2[l]);
+            double* ts = t + static_cast<size_t>(m2[l] - base[l]) * s * s;
+            if (s == kNB) merge2_64_kernel<<<cnt, 256, 0, st>>>(A, n, ts, m2[l]);
+            else merge2_kernel<<<dim3(tiles, cnt), 256, 0, st>>>(A, n, s, ts, m2[l], 0, static_cast<int>(s / kNB));
+            m2[l] = q2;
+          }
         }
         if (m2[l] < m1[l]) break;                       // a pair still waits for its second half
         int q1 = m1[l];
