@@ -152,21 +152,64 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- launch count
+def _inverse_launches(n: int, dones) -> int:
+    """Launches of the factor's inverse: the seeds and the two merge steps of every pair, issued after
+    each group of panels as soon as the columns they need are final (mirrors the host-side schedule;
+    `dones` are the column counts after each group)."""
+    levels = []
+    s = 64
+    while s < n:
+        levels.append({"s": s, "npairs": (n - s + 2 * s - 1) // (2 * s), "slots": max(1, 256 // (2 * s)), "m1": 0, "m2": 0, "rows2": 0})
+        s *= 2
+    count, seeded = 0, 0
+    for done in dones:
+        if done // 64 > seeded:
+            count, seeded = count + 1, done // 64
+        for lv in levels:
+            s = lv["s"]
+            while True:
+                if s > 256:
+                    if lv["m2"] < lv["m1"]:
+                        b0 = lv["m2"] * 2 * s + s
+                        sB = min(s, n - b0)
+                        avail = (min(done, b0 + sB) - b0) // 64
+                        half = s // 128
+                        if avail * 64 < sB:
+                            avail = avail // half * half
+                        if avail > lv["rows2"]:
+                            count, lv["rows2"] = count + 1, avail
+                        if lv["rows2"] * 64 >= sB:
+                            lv["m2"], lv["rows2"] = lv["m2"] + 1, 0
+                else:
+                    q2 = lv["m2"]
+                    while q2 < lv["m1"] and min((q2 + 1) * 2 * s, n) <= done:
+                        q2 += 1
+                    if q2 > lv["m2"]:
+                        count, lv["m2"] = count + 1, q2
+                if lv["m2"] < lv["m1"]:
+                    break
+                q1 = lv["m1"]
+                while q1 < lv["npairs"] and q1 - lv["m1"] < lv["slots"] and q1 * 2 * s + s <= done:
+                    q1 += 1
+                if q1 == lv["m1"]:
+                    break
+                count, lv["m1"] = count + 1, q1
+    return count
+
+
 def launches_hessian_factor(inp: int) -> int:
     """Kernels launched by one Hessian accumulation plus one factor (mirrors the host-side launch logic)."""
     nb = inp // 64
-    factor = 2                                           # damping, build
+    factor = 2 + 1                                       # damping, build; diagonal block 0 (the later ones are factored inside the update kernels)
+    dones = []
     for g0 in range(0, nb, 4):
         g1 = min(g0 + 4, nb)
         for k in range(g0, g1):
             below, inner = nb - k - 1, g1 - k - 1
-            factor += 1 + (1 if below > 0 else 0) + (1 if below > 0 and inner > 0 else 0)
+            factor += (1 if below > 0 else 0) + (1 if below > 0 and inner > 0 else 0)   # panel, in-group update
         factor += (1 if g1 * 64 < inp else 0) + (1 if g1 * 64 + 256 < inp else 0)   # rank-256 update: next group's columns, rest
-    factor += 1 + (2 if inp > 64 else 0)                 # seed, 64-level merges
-    s = 128
-    while s < inp:
-        factor += 2
-        s *= 2
+        dones.append(min(g1 * 64, inp))
+    factor += _inverse_launches(inp, dones)
     factor += 1                                          # emit
     hessian = 2 if inp > 256 else 1
     return hessian + factor

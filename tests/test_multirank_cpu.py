@@ -73,8 +73,11 @@ def test_reference_arm_runs_on_rank_zero_only():
 
 def test_launch_count_matches_the_host_logic():
     import bench
-    # 64-column panels: potrf per panel, panel solve while rows remain below, in-group update while
-    # panels remain in the group, one rank-256 update per finished group with columns to its right
+    # 64-column panels: one launch for diagonal block 0 (the later blocks are factored inside the update
+    # kernels), panel solve while rows remain below, in-group update while panels remain in the group,
+    # one rank-256 update in two launches per finished group with columns to its right; the inverse:
+    # 16 seeds, 2 x 16 launches at level 64, 2 per pair above (3 above half-size 256: the second step
+    # comes in two halves)
     assert bench.launches_per_step(4096, 128) > 0
     n = bench.launches_per_step(4096, 4096)
-    assert n == 325                                    # Hessian 2, RTN 1, scorer 3 + 3, factor 220, GPTQ 96
+    assert n == 366                                    # Hessian 2, RTN 1, scorer 3 + 3, factor 261, GPTQ 96
