@@ -27,6 +27,8 @@ diff_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int g
             adadim_qtensor qa, __nv_bfloat16* __restrict__ Da, adadim_qtensor qb, __nv_bfloat16* __restrict__ Db) {
   const int64_t vecs = in / 8;
   const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  // the product kernel behind this one may be scheduled already: its set-up overlaps this kernel's tail
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (t >= out * vecs) return;
   const int64_t row = t / vecs, col0 = (t % vecs) * 8;
   float w[8];
@@ -76,9 +78,13 @@ diff_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, int g
 // partial is [tiles][2 halves][4]; tiles below `tiles_first` belong to the first scored
 // dimension.  Sums are taken in a fixed order.
 __global__ void __launch_bounds__(256)
-finalize_kernel(const double* __restrict__ partial, int num_tiles, int tiles_first,
+finalize_kernel(const double* partial, int num_tiles, int tiles_first,
                 int first_dim, bool have_second, double* err, int* chosen, int* status_dev) {
   __shared__ double red[2][256];
+  // launched with programmatic serialization behind the product kernel: wait for its completion here.
+  // (`partial` is written by that kernel while this one is already alive, so it is not declared
+  // `const __restrict__`: loads through such a pointer may be moved above the wait.)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   double acc[2] = {0.0, 0.0};
   for (int e = threadIdx.x; e < num_tiles * 2; e += 256) {
     const int tile = e >> 1;
@@ -157,8 +163,20 @@ int score_launch(const void* W, int wdtype, int64_t out, int64_t in, int64_t ldw
   int rc = gram_launch(D, have_second ? D + out * in : nullptr, out, in, H, partial, status_dev, st);
   if (rc != ADADIM_OK) return rc;
   const int tiles = gram_tiles(in);
-  finalize_kernel<<<1, 256, 0, st>>>(partial, tiles * (have_second ? 2 : 1), tiles, first_dim, have_second, err, chosen,
-                                     status_dev);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, finalize_kernel, static_cast<const double*>(partial), tiles * (have_second ? 2 : 1), tiles,
+                           first_dim, have_second, err, chosen, status_dev) != cudaSuccess)
+      return ADADIM_ERR_CUDA;
+  }
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 

@@ -126,6 +126,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // a kernel launched behind this one with programmatic serialization may be scheduled from now on
+  // (it waits for this grid's completion itself before it reads what this grid writes)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
@@ -153,6 +156,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       uint32_t phase = 0;
       int last_phase[STAGES];
       for (int s = 0; s < STAGES; ++s) last_phase[s] = -1;
+      // The scorer's launch is scheduled while the kernel that writes its operands is finishing
+      // (the set-up above overlaps that kernel's tail); the operands are read only from here on.
+      // The H read by the epilogue and everything else this grid touches is older than that kernel.
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int t = blockIdx.x; t < p.num_tiles && !*dead; t += gridDim.x) {
         int rb, cb;
         const int which = MODE == Mode::kGram ? t / p.tiles_per_dim : 0;     // which stacked matrix
@@ -250,6 +257,20 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       tri_coords(MODE == Mode::kGram ? t % p.tiles_per_dim : t, rb, cb);
       bool live = true;
       for (int kc = 0; kc < p.num_k; kc += p.k_chunk) {
+      // Scorer: the H values of the first 32-column chunk are fetched BEFORE the accumulators are
+      // waited for, and every later chunk's while the one before it is being used, so the tensor
+      // pipe (which idles while its only accumulator set is drained) waits for one TMEM read and
+      // 32 multiply-adds per chunk instead of a round trip to L2 each time.
+      float4 h0[8], h1[8];
+      auto load_h = [&](int idx, float4 (&h)[8]) {
+        const int64_t i = static_cast<int64_t>(rb) * 256 + (idx >> 3) * 128 + q * 32 + lane;
+        const int64_t j0 = static_cast<int64_t>(cb) * 256 + (idx & 7) * 32;
+        const float* hrow = p.H + i * p.in + j0;
+#pragma unroll
+        for (int k4 = 0; k4 < 8; ++k4)
+          h[k4] = i < p.in && j0 + k4 * 4 < p.in ? *reinterpret_cast<const float4*>(hrow + k4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      };
+      if (MODE == Mode::kGram) load_h(0, h0);
       live = ptx::mbar_wait(acc_full, acc_phase, dead, p.status_dev);
       if (!live) break;
       ptx::tc_fence_after_sync();
@@ -260,8 +281,30 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         __syncwarp();
       }
       double part[2] = {0.0, 0.0};
+      if (MODE == Mode::kGram) {
+        // sum of H .* (D^T D) over this warp's rows of the tile; tiles below the diagonal stand for
+        // their mirror image too (accumulator entries outside the matrix are zero)
+        auto use_h = [&](int idx, const float4 (&h)[8]) {
+          float v[32];
+          ptx::tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (idx >> 3) * 256 + (idx & 7) * 32, v);
+          float acc = 0.0f;
+#pragma unroll
+          for (int k4 = 0; k4 < 8; ++k4) {
+            acc = fmaf(h[k4].x, v[k4 * 4 + 0], acc); acc = fmaf(h[k4].y, v[k4 * 4 + 1], acc);
+            acc = fmaf(h[k4].z, v[k4 * 4 + 2], acc); acc = fmaf(h[k4].w, v[k4 * 4 + 3], acc);
+          }
+          part[idx >> 3] += static_cast<double>(acc) * (rb == cb ? 1.0 : 2.0);
+        };
 #pragma unroll 1
-      for (int a = 0; a < 2; ++a) {
+        for (int idx = 0; idx < 16; idx += 2) {
+          load_h(idx + 1, h1);
+          use_h(idx, h0);
+          if (idx + 2 < 16) load_h(idx + 2, h0);
+          use_h(idx + 1, h1);
+        }
+      }
+#pragma unroll 1
+      for (int a = 0; a < (MODE == Mode::kGram ? 0 : 2); ++a) {
         const int64_t i = static_cast<int64_t>(rb) * 256 + a * 128 + q * 32 + lane;
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
@@ -289,22 +332,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 ptx::tma_reduce_add_2d(&tmB1, static_cast<int>(j0), static_cast<int>(i0), stage_tile);
                 ptx::bulk_commit();
               }
-            }
-          } else {
-            // sum of H .* (D^T D) over this warp's rows of the tile; tiles below the diagonal
-            // stand for their mirror image too
-            if (i < p.in) {
-              const float* hrow = p.H + i * p.in + j0;
-              float acc = 0.0f;
-#pragma unroll
-              for (int k4 = 0; k4 < 8; ++k4) {
-                if (j0 + k4 * 4 < p.in) {
-                  const float4 h = *reinterpret_cast<const float4*>(hrow + k4 * 4);
-                  acc = fmaf(h.x, v[k4 * 4 + 0], acc); acc = fmaf(h.y, v[k4 * 4 + 1], acc);
-                  acc = fmaf(h.z, v[k4 * 4 + 2], acc); acc = fmaf(h.w, v[k4 * 4 + 3], acc);
-                }
-              }
-              part[a] += static_cast<double>(acc) * (rb == cb ? 1.0 : 2.0);
             }
           }
         }
@@ -403,7 +430,8 @@ hessian_f32_kernel(const float* __restrict__ X, int64_t n_tokens, int64_t in, in
 }
 
 template <Mode MODE>
-int tc_launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const TcParams& p, cudaStream_t st) {
+int tc_launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const TcParams& p, cudaStream_t st,
+              bool chained = false) {
   static int sm_count = 0;
   if (sm_count == 0) {
     int dev = 0;
@@ -413,7 +441,17 @@ int tc_launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1
   ADADIM_CUDA_TRY(cudaFuncSetAttribute(tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(tc_smem_bytes<MODE>())));
   int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
-  tc_kernel<MODE><<<grid, kTcThreads, tc_smem_bytes<MODE>(), st>>>(a, b0, b1, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = tc_smem_bytes<MODE>();
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = chained ? 1 : 0;                      // chained: may start while the launch before it in the stream finishes
+  ADADIM_CUDA_TRY(cudaLaunchKernelEx(&cfg, tc_kernel<MODE>, a, b0, b1, p));
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 
@@ -525,7 +563,7 @@ int gram_launch(const __nv_bfloat16* D0, const __nv_bfloat16* D1, int64_t rows, 
   p.H = const_cast<float*>(H);        // read only in this mode
   p.in = in;
   p.partial = partial;
-  return tc_launch<Mode::kGram>(t0, t1, t0, p, st);
+  return tc_launch<Mode::kGram>(t0, t1, t0, p, st, true);   // behind the kernel that writes D0, D1
 }
 
 int gram_tiles(int64_t in) {
