@@ -18,8 +18,10 @@ def _hessian_f32(X):
     return O.hessian(to_np(X)).astype(np.float32)
 
 
-@pytest.mark.parametrize("n", [64, 128, 256, 704, 1024, 1152, 2048])
+@pytest.mark.parametrize("n", [64, 128, 256, 704, 1024, 1152, 1600, 2048, 2304])
 def test_factor_matches_oracle(n):
+    # 704, 1152, 1600, 2304: a last group of fewer than four panels and merge levels whose last pair is
+    # short or missing; 1600 and 2304 also split the second merge step of their upper levels in two
     kind = "skew" if n == 704 else "normal"
     X = I.make_calib(I.CalibSpec(3 * n, n, "bf16", kind, max(1, n // 128), 30.0, 60.0, seed=31), "cuda")
     Hn = _hessian_f32(X)
