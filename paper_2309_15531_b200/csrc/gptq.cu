@@ -52,24 +52,38 @@ __host__ __device__ constexpr int u_tile_off(int t) { return 32 * (128 * t - 16 
 __host__ __device__ constexpr int u_tile_pitch(int t) { return kBlk - 32 * t; }
 constexpr int kUPacked = u_tile_off(4);              // 10240 doubles
 
+// A CTA fills a strip of 256 columns x kInitRows rows of every copy: lane = 8-column vector of the
+// strip, warp = row lane.  The eight diagonal entries of H that tell dead columns are read once per
+// thread and serve all its rows (they sit in eight different cache lines).
+constexpr int kInitRows = 64;
 template <typename T>
 __global__ void __launch_bounds__(256)
 init_kernel(const T* __restrict__ W, int64_t out, int64_t in, int64_t ldw, const float* __restrict__ H, int ndim,
             double* __restrict__ Wc /* first of ndim consecutive copies of this layer */) {
-  int64_t e = (static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x) * 8;
-  if (e >= out * in) return;
-  int64_t o = e / in, i = e % in;
-  float v[8];
-  load8(W + o * ldw + i, v);
+  const int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + lane * 8;
+  if (i >= in) return;
+  unsigned dead = 0;
 #pragma unroll
   for (int k = 0; k < 8; ++k)
-    if (H[(i + k) * in + (i + k)] == 0.0f) v[k] = 0.0f;        // dead column
-  for (int d = 0; d < ndim; ++d) {
-    double* dst = Wc + static_cast<int64_t>(d) * out * in;
+    if (H[(i + k) * in + (i + k)] == 0.0f) dead |= 1u << k;     // dead column
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kInitRows;
+#pragma unroll 2
+  for (int t = rl; t < kInitRows; t += 8) {
+    const int64_t o = r0 + t;
+    if (o >= out) break;
+    float v[8];
+    load8(W + o * ldw + i, v);
 #pragma unroll
-    for (int k = 0; k < 4; ++k)          // four column pairs of one row of one tile
-      *reinterpret_cast<double2*>(dst + wc_index(o, i + 2 * k, in)) =
-          make_double2(static_cast<double>(v[2 * k]), static_cast<double>(v[2 * k + 1]));
+    for (int k = 0; k < 8; ++k)
+      if ((dead >> k) & 1u) v[k] = 0.0f;
+    for (int d = 0; d < ndim; ++d) {
+      double* dst = Wc + static_cast<int64_t>(d) * out * in;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)          // four column pairs of one row of one tile
+        *reinterpret_cast<double2*>(dst + wc_index(o, i + 2 * k, in)) =
+            make_double2(static_cast<double>(v[2 * k]), static_cast<double>(v[2 * k + 1]));
+    }
   }
 }
 
@@ -733,7 +747,7 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
         if (wdtype == ADADIM_F16) init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, H, perm, nd, dst);
         else init_perm_kernel<<<pb, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, H, perm, nd, dst);
       } else {
-        const unsigned ib = static_cast<unsigned>((y.out * in / 8 + 255) / 256);
+        const dim3 ib(static_cast<unsigned>((in + 255) / 256), static_cast<unsigned>((y.out + kInitRows - 1) / kInitRows));
         if (wdtype == ADADIM_F16) init_kernel<<<ib, 256, 0, st>>>(static_cast<const __half*>(y.W), y.out, in, y.ldw, H, nd, dst);
         else init_kernel<<<ib, 256, 0, st>>>(static_cast<const float*>(y.W), y.out, in, y.ldw, H, nd, dst);
       }
