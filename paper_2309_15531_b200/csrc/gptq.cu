@@ -31,7 +31,7 @@ struct TrailPlan {
 int trail_split_u(const double* U, int64_t in, __nv_bfloat16* u0, __nv_bfloat16* u1, __nv_bfloat16* u2, cudaStream_t st);
 int trail_plan(TrailPlan* plan, double* Wc, int64_t rows_total, int64_t in, const __nv_bfloat16* const e[3],
                const __nv_bfloat16* const u[3]);
-int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int tiles_per_cta, int* status_dev, cudaStream_t st);
+int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_ctas, int* status_dev, cudaStream_t st);
 
 size_t factor_workspace_bytes(int64_t n);
 int factor_launch(const float* H, int64_t n, double percdamp, double* U, int* status_dev, void* workspace,
@@ -771,10 +771,11 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
     if (rc0 != ADADIM_OK) return rc0;
     cudaStream_t chain = fs.chain, side = fs.side;
     cudaEvent_t ev_block = fs.ev_a, ev_rest = fs.ev_b;
-    // the side-stream launches get the SMs that the block kernel leaves free (finer CTAs were
-    // measured slower: every CTA reloads its 96 KB of error pieces and refills the pipeline)
+    // the side-stream launches get the SMs that the block kernel leaves free: one CTA on each, the
+    // launch's tiles dealt out evenly among them; the chain's launch gets the SMs the block kernel
+    // has just left
     const int free_sms = plan.sm_count - slabs % plan.sm_count;
-    const int rest_split = free_sms >= slabs ? free_sms / slabs : 1;
+    const int chain_sms = slabs < plan.sm_count ? slabs : plan.sm_count;
     __nv_bfloat16* ep_base[3] = {a.Ep[0], a.Ep[1], a.Ep[2]};
     bool rest_pending = false;
     for (int i1 = 0; i1 < in; i1 += kBlk) {
@@ -795,12 +796,11 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
         // the next block's columns were last written by the previous block's side-stream launch
         if (rest_pending) ADADIM_CUDA_TRY(cudaStreamWaitEvent(chain, ev_rest, 0));
         rest_pending = false;
-        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, 1, status_dev, chain);
+        rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + kBlk, 1, chain_sms, status_dev, chain);
         if (rc != ADADIM_OK) return rc;
         if (tiles_after > 1) {
           ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_block, 0));
-          rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1,
-                            (tiles_after - 1 + rest_split - 1) / rest_split, status_dev, side);
+          rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1, free_sms, status_dev, side);
           if (rc != ADADIM_OK) return rc;
           ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
           rest_pending = true;

@@ -15,10 +15,13 @@
 // epilogue widens the negated product and hands it to the memory system as an element-wise
 // binary64 add, so the SM never reads W.
 //
-// One CTA owns a 128-row block of the stacked working weights and a range of 128-column
-// tiles.  Its Err pieces (K = 128) stay in shared memory; U pieces stream through a ring of
-// 32-row slabs; two pairs of TMEM accumulators alternate so the read-modify-write of W of one
-// tile overlaps the MMAs of the next.
+// The 128 x 128 tiles of a launch (128-row blocks of the stacked working weights x 128-column
+// tiles) are numbered row block by row block and dealt out in equal contiguous ranges, one per
+// CTA, so that a launch fills exactly the SMs it is given; a range may run from one row block
+// into the next.  The Err pieces of the current row block (K = 128) stay in shared memory and are
+// reloaded when the range crosses into another block; U pieces stream through a ring of 32-row
+// slabs; two pairs of TMEM accumulators alternate so the read-modify-write of W of one tile
+// overlaps the MMAs of the next.
 #include <cuda_bf16.h>
 
 #include "umma.cuh"
@@ -32,9 +35,9 @@ constexpr uint32_t kABytes = 6 * kAPiece;           // 3 pieces x 2 halves
 constexpr int kTileN = 128;
 constexpr uint32_t kBPiece = kTileN * 32 * 2;       // one U piece, 32 k-rows x 128 columns: 8 KB
 constexpr uint32_t kBStage = 3 * kBPiece;           // 24 KB
-constexpr int kBStages = 4;
+constexpr int kBStages = 2;                        // a tile's MMAs are short next to its epilogue: two slabs ahead is enough
 constexpr uint32_t kOutChunk = 32 * 16 * 8;          // one epilogue warp's staging tile: 32 rows x 16 fp64 columns
-constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 8 * kOutChunk + 1024 + 256;
+constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 16 * kOutChunk + 1024 + 256;   // two staging tiles per epilogue warp
 
 struct TrailParams {
   double* Wc;           // stacked working weights, rows_total x in, in the tiled layout of wc_index()
@@ -42,6 +45,7 @@ struct TrailParams {
   int64_t c0;           // first column to update
   int i1;               // first row of U's block
   int ntiles;           // 128-column tiles from c0
+  int mblocks;          // 128-row blocks of the stacked working weights
   int e_row0;           // first row of this block's error pieces (the pieces are kept in two alternating sets)
   int* status_dev;
 };
@@ -55,9 +59,10 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_smem = smem;
   uint8_t* b_smem = smem + kABytes;
-  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][32 rows][128 B]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 8 * kOutChunk);
+  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][2][32 rows][128 B]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 16 * kOutChunk);
   uint64_t* a_full = bars;
+  uint64_t* a_empty = bars + 15;                    // MMA -> TMA: the Err pieces of a finished row block may be overwritten
   uint64_t* b_full = bars + 1;                      // [kBStages]
   uint64_t* b_empty = b_full + kBStages;            // [kBStages]
   uint64_t* acc_full = b_empty + kBStages;          // [2]
@@ -70,14 +75,14 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
   // a kernel launched behind this one with programmatic serialization may be scheduled from now
   // on; it still waits for this grid's completion before it reads anything this grid writes
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // this CTA's tiles: an even share of [0, ntiles)
-  const int per = (p.ntiles + gridDim.x - 1) / gridDim.x;
-  const int t0 = blockIdx.x * per;
-  const int t1 = min(t0 + per, p.ntiles);
-  const int mrow = blockIdx.y * 128;
+  // this CTA's tiles: an even share of [0, mblocks * ntiles), tile g = row block g / ntiles, column tile g % ntiles
+  const int64_t total = static_cast<int64_t>(p.mblocks) * p.ntiles;
+  const int t0 = static_cast<int>(total * blockIdx.x / gridDim.x);
+  const int t1 = static_cast<int>(total * (blockIdx.x + 1) / gridDim.x);
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(a_full, 1);
+    ptx::mbar_init(a_empty, 1);
     for (int s = 0; s < kBStages; ++s) { ptx::mbar_init(&b_full[s], 1); ptx::mbar_init(&b_empty[s], 1); }
     for (int s = 0; s < 2; ++s) { ptx::mbar_init(&acc_full[s], 1); ptx::mbar_init(&acc_empty[s], 8); }
     ptx::mbar_init(drain, 1);
@@ -97,15 +102,23 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
     if (lane == 0 && t0 < t1) {
       const CUtensorMap* tmE[3] = {&tmE0, &tmE1, &tmE2};
       const CUtensorMap* tmU[3] = {&tmU0, &tmU1, &tmU2};
-      ptx::mbar_arrive_expect_tx(a_full, kABytes);
-      for (int pc = 0; pc < 3; ++pc)
-        for (int kh = 0; kh < 2; ++kh)
-          ptx::tma_load_2d(a_smem + (pc * 2 + kh) * kAPiece, tmE[pc], kh * 64, p.e_row0 + mrow, a_full);
       int stage = 0;
       uint32_t phase = 0;
       int last_phase[kBStages];
       for (int s = 0; s < kBStages; ++s) last_phase[s] = -1;
-      for (int t = t0; t < t1 && !*dead; ++t) {
+      int rb_now = -1, a_loads = 0;
+      for (int g = t0; g < t1 && !*dead; ++g) {
+        const int rb = g / p.ntiles, t = g % p.ntiles;
+        if (rb != rb_now) {
+          // Err pieces of the next row block, once the MMAs that read the previous ones are done
+          if (a_loads > 0 && !ptx::mbar_wait(a_empty, static_cast<uint32_t>((a_loads - 1) & 1), dead, p.status_dev)) break;
+          ptx::mbar_arrive_expect_tx(a_full, kABytes);
+          for (int pc = 0; pc < 3; ++pc)
+            for (int kh = 0; kh < 2; ++kh)
+              ptx::tma_load_2d(a_smem + (pc * 2 + kh) * kAPiece, tmE[pc], kh * 64, p.e_row0 + rb * 128, a_full);
+          rb_now = rb;
+          ++a_loads;
+        }
         const int col = static_cast<int>(p.c0) + t * kTileN;
         for (int kc = 0; kc < 4; ++kc) {
           if (!ptx::mbar_wait(&b_empty[stage], phase ^ 1u, dead, p.status_dev)) break;
@@ -121,7 +134,7 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
       if (*dead) {
         // a wait ran out somewhere: let the copies already issued land before shared memory goes away
         const long long c0 = clock64();
-        while (!ptx::mbar_try_wait(a_full, 0) && clock64() - c0 < ptx::kWaitLimit) {}
+        while (a_loads > 0 && !ptx::mbar_try_wait(a_full, static_cast<uint32_t>((a_loads - 1) & 1)) && clock64() - c0 < ptx::kWaitLimit) {}
         for (int s = 0; s < kBStages; ++s) {
           if (last_phase[s] < 0) continue;
           const long long c1 = clock64();
@@ -134,11 +147,17 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
       constexpr uint32_t idesc = ptx::idesc_bf16(128, kTileN, false, true);
       constexpr uint64_t adesc = ptx::smem_desc_sw128(16, 1024);          // K-major, 8-row groups 1024 B apart
       constexpr uint64_t bdesc = ptx::smem_desc_sw128(32 * 128, 1024);    // MN-major, 64-column blocks 4 KB apart
-      bool ok = ptx::mbar_wait(a_full, 0, dead, p.status_dev);
-      int stage = 0;
+      bool ok = true;
+      int stage = 0, rb_now = -1, a_seen = 0;
       uint32_t phase = 0, acc_phase[2] = {0, 0};
-      for (int t = t0; t < t1 && ok; ++t) {
-        const int buf = (t - t0) & 1;
+      for (int g = t0; g < t1 && ok; ++g) {
+        const int rb = g / p.ntiles;
+        if (rb != rb_now) {
+          if (!ptx::mbar_wait(a_full, static_cast<uint32_t>(a_seen & 1), dead, p.status_dev)) break;
+          rb_now = rb;
+          ++a_seen;
+        }
+        const int buf = (g - t0) & 1;
         if (!ptx::mbar_wait(&acc_empty[buf], acc_phase[buf] ^ 1u, dead, p.status_dev)) break;
         ptx::tc_fence_after_sync();
         for (int kc = 0; kc < 4; ++kc) {
@@ -166,6 +185,7 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
         if (!ok) break;
         ptx::mma_commit(&acc_full[buf]);
         acc_phase[buf] ^= 1u;
+        if (g + 1 < t1 && (g + 1) / p.ntiles != rb) ptx::mma_commit(a_empty);    // this row block's Err pieces are free once these MMAs are done
       }
       if (*dead) {
         ptx::mma_commit(drain);
@@ -181,13 +201,13 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
     // operation as W - p), so the epilogue only issues writes.
     const int q = warp & 3, half = (warp - 2) >> 2;
     uint32_t acc_phase[2] = {0, 0};
-    uint8_t* stage_tile = out_smem + (warp - 2) * kOutChunk;
-    uint8_t* my_row = stage_tile + lane * 128;        // this lane's row of the staging tile
-    // first tile of this warp's rows and of the launch's first column
-    double* wtile = p.Wc + (static_cast<int64_t>((mrow + q * 32) / kWcTileRows) * (p.in / kWcTileCols) +
-                            (p.c0 + half * 64) / kWcTileCols) * kWcTileElems;
-    for (int t = t0; t < t1; ++t) {
-      const int buf = (t - t0) & 1;
+    uint8_t* stage_tiles = out_smem + (warp - 2) * 2 * kOutChunk;    // two staging tiles, used in turn: two adds in flight
+    for (int g = t0; g < t1; ++g) {
+      const int rb = g / p.ntiles, t = g % p.ntiles;
+      const int buf = (g - t0) & 1;
+      // first tile of this warp's rows of the row block and of the launch's first column
+      double* wtile = p.Wc + (static_cast<int64_t>((rb * 128 + q * 32) / kWcTileRows) * (p.in / kWcTileCols) +
+                              (p.c0 + half * 64) / kWcTileCols) * kWcTileElems;
       if (!ptx::mbar_wait(&acc_full[buf], acc_phase[buf], dead, p.status_dev)) break;
       ptx::tc_fence_after_sync();
 #pragma unroll
@@ -197,7 +217,9 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
         ptx::tmem_ld16_nowait(taddr, v);
         ptx::tmem_ld16_nowait(taddr + kTileN, v2);
         ptx::tmem_ld_wait();
-        if (lane == 0) ptx::bulk_wait_read();         // the previous add has finished reading the staging tile
+        uint8_t* stage_tile = stage_tiles + (c & 1) * kOutChunk;
+        uint8_t* my_row = stage_tile + lane * 128;    // this lane's row of the staging tile
+        if (lane == 0) ptx::bulk_wait_read_but_one();  // the add before the previous one has finished reading this staging tile
         __syncwarp();
 #pragma unroll
         for (int k = 0; k < 8; ++k) {                  // column pair k of the row sits at pair position k ^ (row % 8)
@@ -314,25 +336,24 @@ int trail_plan(TrailPlan* plan, double* Wc, int64_t rows_total, int64_t in, cons
   return ADADIM_OK;
 }
 
-// Updates `ntiles` 128-column tiles starting at column c0 with the errors of the block whose first
-// column is i1 (error set i1/128 & 1); every CTA takes about `tiles_per_cta` tiles of one 128-row
-// block.  Small CTAs let a launch that runs beside higher-priority kernels use whatever SMs are
-// idle and hand them back quickly.
-int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int tiles_per_cta, int* status_dev, cudaStream_t st) {
+// Updates `ntiles` 128-column tiles starting at column c0, in every 128-row block, with the errors of
+// the block whose first column is i1 (error set i1/128 & 1), on at most `max_ctas` CTAs (one per SM:
+// the count of SMs the caller leaves to this launch).
+int trail_launch(const TrailPlan& plan, int i1, int64_t c0, int ntiles, int max_ctas, int* status_dev, cudaStream_t st) {
   TrailParams p;
   p.Wc = plan.Wc;
   p.in = plan.in;
   p.c0 = c0;
   p.i1 = i1;
   p.ntiles = ntiles;
+  p.mblocks = static_cast<int>(plan.rows_total / 128);
   p.e_row0 = static_cast<int>(((i1 / 128) & 1) * plan.rows_total);
   p.status_dev = status_dev;
   if (p.ntiles <= 0) return ADADIM_OK;
-  const int mblocks = static_cast<int>(plan.rows_total / 128);
-  int nsplit = (ntiles + tiles_per_cta - 1) / tiles_per_cta;
-  if (nsplit < 1) nsplit = 1;
-  trail_kernel<<<dim3(nsplit, mblocks), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],
-                                                                      plan.u[1], plan.u[2], p);
+  const int64_t total = static_cast<int64_t>(p.mblocks) * ntiles;
+  const int ctas = static_cast<int>(total < max_ctas ? total : max_ctas);
+  trail_kernel<<<dim3(static_cast<unsigned>(ctas < 1 ? 1 : ctas)), kThreads, kSmemBytes, st>>>(plan.e[0], plan.e[1], plan.e[2], plan.u[0],
+                                                                                                plan.u[1], plan.u[2], p);
   return cudaGetLastError() == cudaSuccess ? ADADIM_OK : ADADIM_ERR_CUDA;
 }
 
