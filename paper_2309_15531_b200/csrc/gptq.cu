@@ -800,7 +800,12 @@ int gptq_launch(const GptqLayer* layers, int n_layers, int wdtype, int64_t in, c
         if (rc != ADADIM_OK) return rc;
         if (tiles_after > 1) {
           ADADIM_CUDA_TRY(cudaStreamWaitEvent(side, ev_block, 0));
-          rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1, free_sms, status_dev, side);
+          // On the free SMs alone the launch runs beside the next block kernel.  Where the block kernel
+          // leaves fewer than half of the SMs (128 slabs on 148 SMs: 20), the launch gets all of them
+          // instead and the two alternate (8192 x 28672 in both dimensions: 748 ms on the 20 free SMs,
+          // 187 ms on all; 64 slabs x 11008 columns: 15.3 ms on the 84 free SMs, 16.1 ms on all).
+          const bool all = 2 * free_sms < plan.sm_count;
+          rc = trail_launch(plan, i1, static_cast<int64_t>(i1) + 2 * kBlk, tiles_after - 1, all ? plan.sm_count : free_sms, status_dev, side);
           if (rc != ADADIM_OK) return rc;
           ADADIM_CUDA_TRY(cudaEventRecord(ev_rest, side));
           rest_pending = true;
