@@ -35,9 +35,9 @@ constexpr uint32_t kABytes = 6 * kAPiece;           // 3 pieces x 2 halves
 constexpr int kTileN = 128;
 constexpr uint32_t kBPiece = kTileN * 32 * 2;       // one U piece, 32 k-rows x 128 columns: 8 KB
 constexpr uint32_t kBStage = 3 * kBPiece;           // 24 KB
-constexpr int kBStages = 2;                        // a tile's MMAs are short next to its epilogue: two slabs ahead is enough
+constexpr int kBStages = 4;
 constexpr uint32_t kOutChunk = 32 * 16 * 8;          // one epilogue warp's staging tile: 32 rows x 16 fp64 columns
-constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 16 * kOutChunk + 1024 + 256;   // two staging tiles per epilogue warp
+constexpr size_t kSmemBytes = kABytes + kBStages * kBStage + 8 * kOutChunk + 1024 + 256;
 
 struct TrailParams {
   double* Wc;           // stacked working weights, rows_total x in, in the tiled layout of wc_index()
@@ -59,8 +59,8 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_smem = smem;
   uint8_t* b_smem = smem + kABytes;
-  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][2][32 rows][128 B]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 16 * kOutChunk);
+  uint8_t* out_smem = b_smem + kBStages * kBStage;  // [8 warps][32 rows][128 B]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 8 * kOutChunk);
   uint64_t* a_full = bars;
   uint64_t* a_empty = bars + 15;                    // MMA -> TMA: the Err pieces of a finished row block may be overwritten
   uint64_t* b_full = bars + 1;                      // [kBStages]
@@ -201,7 +201,8 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
     // operation as W - p), so the epilogue only issues writes.
     const int q = warp & 3, half = (warp - 2) >> 2;
     uint32_t acc_phase[2] = {0, 0};
-    uint8_t* stage_tiles = out_smem + (warp - 2) * 2 * kOutChunk;    // two staging tiles, used in turn: two adds in flight
+    uint8_t* stage_tile = out_smem + (warp - 2) * kOutChunk;
+    uint8_t* my_row = stage_tile + lane * 128;        // this lane's row of the staging tile
     for (int g = t0; g < t1; ++g) {
       const int rb = g / p.ntiles, t = g % p.ntiles;
       const int buf = (g - t0) & 1;
@@ -217,9 +218,7 @@ trail_kernel(const __grid_constant__ CUtensorMap tmE0, const __grid_constant__ C
         ptx::tmem_ld16_nowait(taddr, v);
         ptx::tmem_ld16_nowait(taddr + kTileN, v2);
         ptx::tmem_ld_wait();
-        uint8_t* stage_tile = stage_tiles + (c & 1) * kOutChunk;
-        uint8_t* my_row = stage_tile + lane * 128;    // this lane's row of the staging tile
-        if (lane == 0) ptx::bulk_wait_read_but_one();  // the add before the previous one has finished reading this staging tile
+        if (lane == 0) ptx::bulk_wait_read();         // the previous add has finished reading the staging tile
         __syncwarp();
 #pragma unroll
         for (int k = 0; k < 8; ++k) {                  // column pair k of the row sits at pair position k ^ (row % 8)

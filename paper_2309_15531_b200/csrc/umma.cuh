@@ -119,8 +119,6 @@ __device__ __forceinline__ void bulk_reduce_add_f64(double* dst, const void* src
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // until the committed groups have finished READING shared memory (the source may be reused)
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// all but the latest committed group have finished reading their shared-memory source
-__device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 // until the committed groups are complete
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // orders this thread's generic-proxy shared-memory writes before later async-proxy (TMA) reads
