@@ -16,8 +16,9 @@
  *     adadim_score_select_static); inputs are never modified.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *     stream).  No entry point synchronizes; results are valid once the stream has run.
- *     adadim_cholesky_inverse_factor and the two GPTQ entry points overlap parts of their work
- *     on two streams of their own, which they create on entry and release before returning;
+ *     adadim_cholesky_inverse_factor and the GPTQ entry points overlap parts of their work
+ *     on streams of their own (two; four in the factor), which they create on entry and release
+ *     before returning;
  *     that work starts after everything already enqueued on `cuda_stream` and is joined back
  *     into it, so to the caller these calls are ordered on `cuda_stream` like the others.
  *   - The return value is an adadim_status.  Argument errors are found on the host before
